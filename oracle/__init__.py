@@ -1,0 +1,162 @@
+"""Python face of the CPU oracle (oracle/rocket_oracle.c).
+
+TEST INFRASTRUCTURE ONLY: importable from tests/, from the smoke check and from the
+benchmark's CPU-baseline leg.  The product package never imports it, and it never
+imports the product package.  Functions take a rocket_inputs.KernelParams (plain numpy
+arrays) and numpy inputs, and return numpy float64 / integer arrays.
+"""
+import ctypes
+import os
+import subprocess
+from types import SimpleNamespace
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "rocket_oracle.c")
+_LIB = os.path.join(_HERE, "_build", "librocket_oracle.so")
+_lib = None
+
+
+def build(force=False):
+    """Compile the oracle with gcc (-O2, OpenMP).  Returns the path of the shared object."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        os.makedirs(os.path.dirname(_LIB), exist_ok=True)
+        tmp = _LIB + ".%d.tmp" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
+                               "-ffp-contract=off", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _CParams(ctypes.Structure):
+    _fields_ = [("K", ctypes.c_int), ("C", ctypes.c_int), ("L", ctypes.c_int),
+                ("length", ctypes.c_void_p), ("dilation", ctypes.c_void_p),
+                ("padding", ctypes.c_void_p), ("num_channels", ctypes.c_void_p),
+                ("channel_idx", ctypes.c_void_p), ("weights", ctypes.c_void_p),
+                ("bias", ctypes.c_void_p), ("channel_offset", ctypes.c_void_p),
+                ("weight_offset", ctypes.c_void_p)]
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        lib.rocket_oracle_conv.restype = ctypes.c_int64
+        lib.rocket_oracle_num_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _ptr(a):
+    return a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
+
+
+def _cparams(p):
+    """Pack a KernelParams into the C struct; returns (struct, keepalive list)."""
+    arrs = dict(
+        length=np.ascontiguousarray(p.length, np.int32), dilation=np.ascontiguousarray(p.dilation, np.int32),
+        padding=np.ascontiguousarray(p.padding, np.int32),
+        num_channels=np.ascontiguousarray(p.num_channels, np.int32),
+        channel_idx=np.ascontiguousarray(p.channel_idx, np.int32),
+        weights=np.ascontiguousarray(p.weights, np.float32), bias=np.ascontiguousarray(p.bias, np.float32),
+        channel_offset=np.ascontiguousarray(p.channel_offset, np.int64),
+        weight_offset=np.ascontiguousarray(p.weight_offset, np.int64))
+    s = _CParams(K=p.K, C=p.C, L=p.L, **{k: v.ctypes.data for k, v in arrs.items()})
+    return s, arrs
+
+
+def _check_x(p, X):
+    X = np.ascontiguousarray(X, dtype=np.float32)
+    if X.ndim != 3 or X.shape[1] != p.C or X.shape[2] != p.L:
+        raise ValueError("X must be [N, %d, %d]" % (p.C, p.L))
+    return X
+
+
+def num_threads():
+    return int(_load().rocket_oracle_num_threads())
+
+
+def set_threads(t):
+    _load().rocket_oracle_set_threads(ctypes.c_int(int(t)))
+
+
+def conv(p, X, n, k):
+    """z[0..L_out) of kernel k on example n, float64."""
+    lib = _load()
+    X = _check_x(p, X)
+    s, keep = _cparams(p)
+    nout = lib.rocket_oracle_conv(ctypes.byref(s), _ptr(X), ctypes.c_int(n), ctypes.c_int(k), None)
+    z = np.empty(max(int(nout), 0), dtype=np.float64)
+    lib.rocket_oracle_conv(ctypes.byref(s), _ptr(X), ctypes.c_int(n), ctypes.c_int(k), _ptr(z))
+    return z
+
+
+def forward_pairs(p, X, pair_n, pair_k, lam=1.0, shift=3.0, amb_eps=1e-5):
+    """Pooled features for explicit (example, kernel) pairs.
+
+    Returns a namespace of 1-D arrays: ppv, max, soft (float64), argmax (int32),
+    pos_eps, amb (int64), gap (float64), out_len (int64).
+    """
+    lib = _load()
+    X = _check_x(p, X)
+    pn = np.ascontiguousarray(pair_n, np.int32)
+    pk = np.ascontiguousarray(pair_k, np.int32)
+    if pn.shape != pk.shape or pn.ndim != 1:
+        raise ValueError("pair_n and pair_k must be 1-D and of equal length")
+    if len(pn) and (pn.min() < 0 or pn.max() >= X.shape[0] or pk.min() < 0 or pk.max() >= p.K):
+        raise ValueError("pair index out of range")
+    P = len(pn)
+    out = SimpleNamespace(ppv=np.empty(P), max=np.empty(P), soft=np.empty(P), argmax=np.empty(P, np.int32),
+                          pos_eps=np.empty(P, np.int64), amb=np.empty(P, np.int64), gap=np.empty(P))
+    s, keep = _cparams(p)
+    lib.rocket_oracle_forward_pairs(ctypes.byref(s), _ptr(X), ctypes.c_int64(P), _ptr(pn), _ptr(pk),
+                                    ctypes.c_double(lam), ctypes.c_double(shift), ctypes.c_double(amb_eps),
+                                    _ptr(out.ppv), _ptr(out.max), _ptr(out.soft), _ptr(out.argmax),
+                                    _ptr(out.pos_eps), _ptr(out.amb), _ptr(out.gap))
+    out.out_len = p.out_len[pk]
+    return out
+
+
+def forward(p, X, lam=1.0, shift=3.0, amb_eps=1e-5):
+    """Pooled features for every (example, kernel): each field reshaped to [N, K]."""
+    N = np.asarray(X).shape[0]
+    pn = np.repeat(np.arange(N, dtype=np.int32), p.K)
+    pk = np.tile(np.arange(p.K, dtype=np.int32), N)
+    out = forward_pairs(p, X, pn, pk, lam, shift, amb_eps)
+    for name, v in vars(out).items():
+        setattr(out, name, v.reshape(N, p.K))
+    return out
+
+
+def features_hard(out):
+    """Interleave (PPV_k, MAX_k) into [N, 2K], the layout of the library's feature matrix."""
+    return np.stack([out.ppv, out.max], axis=-1).reshape(out.ppv.shape[0], -1)
+
+
+def features_soft(out):
+    return np.stack([out.soft, out.max], axis=-1).reshape(out.soft.shape[0], -1)
+
+
+def backward(p, X, g, argmax, lam=1.0, shift=3.0, examples=None, kernels=None):
+    """Gradients (dW ragged float64, db float64[K]) of sum(g * features_soft).
+
+    g: [N, 2K] float32 interleaved (gP, gM); argmax: [N, K] int32.  examples / kernels
+    restrict the sum over n and the kernels computed (others are left at zero).
+    """
+    lib = _load()
+    X = _check_x(p, X)
+    N = X.shape[0]
+    g = np.ascontiguousarray(g, np.float32)
+    argmax = np.ascontiguousarray(argmax, np.int32)
+    if g.shape != (N, 2 * p.K) or argmax.shape != (N, p.K):
+        raise ValueError("g must be [N, 2K] and argmax [N, K]")
+    ex = np.arange(N, dtype=np.int32) if examples is None else np.ascontiguousarray(examples, np.int32)
+    ks = np.arange(p.K, dtype=np.int32) if kernels is None else np.ascontiguousarray(kernels, np.int32)
+    dW = np.zeros(len(p.weights), dtype=np.float64)
+    db = np.zeros(p.K, dtype=np.float64)
+    s, keep = _cparams(p)
+    lib.rocket_oracle_backward(ctypes.byref(s), _ptr(X), ctypes.c_int(len(ex)), _ptr(ex), ctypes.c_int(len(ks)),
+                               _ptr(ks), ctypes.c_double(lam), ctypes.c_double(shift), _ptr(g), _ptr(argmax),
+                               _ptr(dW), _ptr(db))
+    return dW, db
