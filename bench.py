@@ -1,0 +1,327 @@
+#!/usr/bin/env python
+"""Benchmark of the ROCKET transform hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one hard transform (PPV + max) of the paper-scale batch: 60 examples x 20 channels x
+50,000 steps through 10,000 random kernels, the workload the metric is quoted on.  The same run
+also times the soft forward and the soft backward on the training-pass shape (32 examples) and
+reports them under "passes".  Prints ONE JSON line on rank 0.
+
+Multi-GPU: (example, kernel) pairs are independent, so ranks each transform their own batch of
+60 examples (weak scaling, no data-path collective); torch.distributed is used for the barrier
+and the max-over-ranks of the timings only.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "ROCKET transform examples/s at 20ch x 50k, 10k kernels; % of FP32 FMA peak"
+UNIT = "examples/s"
+WORKLOAD = dict(N=60, C=20, L=50000, K=10000)        # paper-scale inference batch
+TRAIN = dict(N=32, C=20, L=50000, K=10000)           # soft forward + backward shape
+PARAM_SEED, DATA_SEED, GRAD_SEED = 8527, 2301, 527
+LAMBDA, SHIFT = 10.0, 3.0
+
+# DRAM bytes (read + write) of one launch of the dominant kernel, from the committed ncu capture
+# (profiles/); None until a capture of the current kernel exists.
+NCU_DRAM_BYTES_PER_LAUNCH = None
+
+
+def fp32_peak_tflops(sm_count, sm_mhz):
+    """FP32 FMA peak: SMs x 128 lanes x 2 flop x clock."""
+    return sm_count * 128 * 2 * sm_mhz * 1e6 / 1e12
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return json.load(f)
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def run_reference(args, rank):
+    """The CPU oracle, as it stands, on the machine's host cores: a bounded sample of the workload per step."""
+    if rank != 0:
+        return
+    import oracle
+    from rocket_inputs import ar1_spike_series, generate_kernels
+    w = WORKLOAD
+    kp = generate_kernels(PARAM_SEED, w["K"], w["C"], w["L"])
+    X = ar1_spike_series(DATA_SEED, 1, w["C"], w["L"])
+    ks = np.sort(np.random.default_rng(1).choice(w["K"], args.ref_kernels, replace=False)).astype(np.int32)
+    pn = np.zeros(len(ks), np.int32)
+    # an example costs sum_k flops(k); the sample's share of that cost scales its time to one example
+    flops_k = 2.0 * kp.length * kp.num_channels * kp.out_len
+    share = flops_k[ks].sum() / flops_k.sum()
+    oracle.forward_pairs(kp, X, pn[:8], ks[:8])
+    times = []
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        oracle.forward_pairs(kp, X, pn, ks)
+        if it >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    per_example = float(np.mean(times)) / share
+    value = 1.0 / per_example
+    cores = oracle.num_threads()
+    sample = "1 example x %d of %d kernels per step (%.2f%% of an example's conv flop), scaled by flop share" % (
+        len(ks), w["K"], 100 * share)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(times)),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "N=60 x C=20 x L=50000, K=10000 multivariate kernels, hard PPV + max (config 2)",
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def cpu_baseline(kp, X1, seconds_budget=20.0):
+    """Times the oracle on a bounded sample of the workload (rank 0, N=1 only)."""
+    import oracle
+    K = kp.K
+    flops_k = 2.0 * kp.length * kp.num_channels * kp.out_len
+    rng = np.random.default_rng(1)
+    probe = np.sort(rng.choice(K, 16, replace=False)).astype(np.int32)
+    t0 = time.perf_counter()
+    oracle.forward_pairs(kp, X1, np.zeros(len(probe), np.int32), probe)
+    rate = flops_k[probe].sum() / max(time.perf_counter() - t0, 1e-6)      # flop/s, rough
+    nk = int(np.clip(seconds_budget * rate / flops_k.mean(), 32, K))
+    ks = np.sort(rng.choice(K, nk, replace=False)).astype(np.int32)
+    t0 = time.perf_counter()
+    oracle.forward_pairs(kp, X1, np.zeros(nk, np.int32), ks)
+    dt = time.perf_counter() - t0
+    share = flops_k[ks].sum() / flops_k.sum()
+    return {"value": share / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "1 example x %d of %d kernels (%.2f%% of an example's conv flop) in %.1f s, scaled by flop share"
+                      % (nk, K, 100 * share, dt)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-kernels", type=int, default=2000, help="kernels per step of the reference arm's sample")
+    ap.add_argument("--skip-passes", action="store_true", help="skip the soft forward / backward timings")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--small", action="store_true", help="profiling case: N=8 examples (160 MB... of input)")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2301_08527_b200 as rk
+    from paper_2301_08527_b200 import binding
+    from rocket_inputs import ar1_spike_series, generate_kernels, normal_array
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the transform has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(v):
+        if world == 1:
+            return v
+        t = torch.tensor([v], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    w = dict(WORKLOAD)
+    if args.small:
+        w["N"] = 8
+    props = torch.cuda.get_device_properties(local_rank)
+    params = rk.RocketParams.generate(PARAM_SEED, w["K"], w["C"], w["L"])
+    flops_ex, outputs_ex = params.work()
+
+    # each rank owns its own batch (weak scaling): different data seed per rank
+    X_host = torch.from_numpy(ar1_spike_series(DATA_SEED + 1000 * rank, w["N"], w["C"], w["L"])).pin_memory()
+    X = X_host.cuda()
+    feat = torch.empty((w["N"], 2 * w["K"]), dtype=torch.float32, device="cuda")
+    feat_host = torch.empty((w["N"], 2 * w["K"]), dtype=torch.float32).pin_memory()
+    stream = torch.cuda.current_stream()
+
+    def time_steps(fn, steps, warmup):
+        """CUDA-event time of `steps` calls on the launching stream, after `warmup` calls; seconds."""
+        for _ in range(warmup):
+            fn()
+        barrier()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        evs[0].record(stream)
+        for i in range(steps):
+            fn()
+            evs[i + 1].record(stream)
+        barrier()
+        per = [evs[i].elapsed_time(evs[i + 1]) * 1e-3 for i in range(steps)]
+        return evs[0].elapsed_time(evs[-1]) * 1e-3, per
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    launches0 = rk.kernel_launch_count()
+    if sampler:
+        sampler.start()
+    total_s, per_step = time_steps(lambda: rk.rocket_transform(params, X, out=feat), args.steps, args.warmup)
+    clocks = sampler.stop() if sampler else None
+    launches = rk.kernel_launch_count() - launches0
+    launches_timed = launches * args.steps // (args.steps + args.warmup)
+    total_s = max_over_ranks(total_s)
+    ms_per_step = 1e3 * total_s / args.steps
+    value = world * w["N"] * args.steps / total_s
+
+    # end to end through the host-buffer entry point: H2D of X and D2H of the features inside the timing
+    def e2e_step():
+        binding.rocket_transform_host(params, X_host, feat_host)
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    e2e_steps = max(3, args.steps // 2)
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = max_over_ranks(time.perf_counter() - t0)
+    e2e = {"value": world * w["N"] * e2e_steps / e2e_s, "unit": UNIT,
+           "h2d_bytes_per_step": X_host.numel() * 4, "d2h_bytes_per_step": feat_host.numel() * 4,
+           "steps": e2e_steps, "api": "rocket_transform_host (pinned host buffers)"}
+
+    # roofline of the dominant kernel: the fused hard-transform kernel, one launch per step
+    kernel_s = float(np.mean(per_step))
+    achieved = flops_ex * w["N"] / kernel_s / 1e12
+    peaks = measured_peaks()
+    sm_max = (peaks or {}).get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
+    peak = fp32_peak_tflops(props.multi_processor_count, sm_max)
+    roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "traffic": NCU_DRAM_BYTES_PER_LAUNCH,
+                "peak_source": "%d SMs x 128 FP32 lanes x 2 flop x %.0f MHz (max SM clock, %s)" % (
+                    props.multi_processor_count, sm_max, "MEASURED_PEAKS.json" if peaks else "nvidia-smi / nominal"),
+                "flop_count": "2*len*channels*L_out per kernel per example = %.4g flop/example" % flops_ex,
+                "pooling_ops_per_example": 2.0 * outputs_ex}
+    if clocks and clocks.get("sm_mhz"):
+        roofline["frac_at_observed_clock"] = achieved / fp32_peak_tflops(props.multi_processor_count, clocks["sm_mhz"])
+
+    passes = None
+    if not args.skip_passes and not args.small:
+        t = TRAIN
+        Xt = X[: t["N"]]
+        g = torch.from_numpy(normal_array(GRAD_SEED, (t["N"], 2 * t["K"]))).cuda()
+        sfeat = torch.empty((t["N"], 2 * t["K"]), dtype=torch.float32, device="cuda")
+        arg = torch.empty((t["N"], t["K"]), dtype=torch.int32, device="cuda")
+        dW = torch.empty((params.n_weights,), dtype=torch.float32, device="cuda")
+        db = torch.empty((t["K"],), dtype=torch.float32, device="cuda")
+        psteps = max(2, args.steps // 3)
+        s_soft, _ = time_steps(lambda: rk.rocket_transform_soft(params, Xt, LAMBDA, SHIFT, out=sfeat, argmax_out=arg),
+                               psteps, 3)
+        s_bwd, _ = time_steps(lambda: rk.rocket_transform_soft_backward(params, Xt, LAMBDA, SHIFT, g, arg, dW, db),
+                              psteps, 3)
+        s_soft, s_bwd = max_over_ranks(s_soft) / psteps, max_over_ranks(s_bwd) / psteps
+        passes = {
+            "shape": "N=32 x C=20 x L=50000, K=10000 (config 3), lambda=%g, shift=%g" % (LAMBDA, SHIFT),
+            "soft_forward": {"examples_per_s": world * t["N"] / s_soft, "ms": 1e3 * s_soft,
+                             "conv_tflops": flops_ex * t["N"] / s_soft / 1e12},
+            "soft_backward": {"examples_per_s": world * t["N"] / s_bwd, "ms": 1e3 * s_bwd,
+                              "conv_tflops": 2 * flops_ex * t["N"] / s_bwd / 1e12,
+                              "flop_count": "4*len*channels*L_out (recompute z + dW)"},
+        }
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.skip_cpu_baseline:
+        kp = generate_kernels(PARAM_SEED, w["K"], w["C"], w["L"])
+        cpu = cpu_baseline(kp, X_host[:1].numpy())
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "N=%d x C=%d x L=%d fp32, K=%d multivariate kernels, hard PPV + max (config 2)%s" % (
+                           w["N"], w["C"], w["L"], w["K"], " [reduced N for profiling]" if args.small else ""),
+                       "examples_per_gpu": w["N"], "l2": "inputs larger than L2 (%.0f MB per batch)" % (
+                           X_host.numel() * 4 / 1e6), "timing": "CUDA events on the launching stream",
+                       "seeds": {"params": PARAM_SEED, "data": DATA_SEED}},
+            "conv_tflops": achieved, "pct_fp32_peak": 100 * achieved / peak,
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_timed,
+            "clocks": clocks, "passes": passes,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,168 @@
+/*
+ * rocket.h - C ABI of the B200 ROCKET transform library.
+ *
+ * The library computes the random-convolution transform of ROCKET (Section 3 of "Making the
+ * exceptionally fast ROCKET model faster"): K random dilated, optionally "same"-padded,
+ * multichannel 1-D convolution kernels are applied to a batch of series X[N][C][L] and each
+ * kernel's output is reduced on the fly to two pooled features, so the N*K*L_out convolution
+ * outputs never leave the chip.
+ *
+ *   z[n,k,i] = b_k + sum_{q<m_k} sum_{j<len_k} W_k[q][j] * xpad[n, S_k[q], i - p_k + j*d_k]
+ *              for 0 <= i < L_out,k = L + 2 p_k - (len_k - 1) d_k, xpad = 0 outside [0, L)
+ *   PPV      = (1/L_out) #{ i : z_i > 0 }                               (Eq. 1-2)
+ *   MAX      = max_i z_i                                                (Section 3, step (2))
+ *   softPPV  = (1/L_out) sum_i 1 / (1 + exp(-(lambda z_i + shift)))     (Eq. 3-4)
+ *
+ * Conventions common to every call
+ *   - Pointers named *_dev are device pointers; pointers named *_host and all other pointers
+ *     are host pointers.  A handle binds to the device that is current at its first device
+ *     call (its parameters are uploaded then, once) and every later call with that handle
+ *     runs on that device.  Creating, inspecting and destroying a handle needs no device.
+ *   - X is dense row-major [N][C][L] fp32.  Features are fp32 [N][2K], interleaved:
+ *     feat[n][2k] = PPV_k (or softPPV_k), feat[n][2k+1] = MAX_k.
+ *   - Kernel parameters are ragged: kernel k owns num_channels[k] consecutive entries of
+ *     channel_idx and num_channels[k]*length[k] consecutive weights, row-major [q][j].
+ *   - Device calls enqueue work on the caller's stream (a cudaStream_t passed as void*, NULL =
+ *     the legacy default stream) and return without synchronising.  Outputs are fully
+ *     overwritten.  The caller owns every buffer it passes; the library owns the handle and
+ *     the workspace inside it.  Two calls that use the same handle must be ordered on the
+ *     device (same stream, or an event between them): they share the handle's workspace.
+ *   - Every function returns a rocket_status_t (0 = success).  Argument errors are detected
+ *     on the host before anything is launched and leave the outputs untouched.  Nothing
+ *     aborts and nothing throws across this boundary.  There is no CPU fallback: without a
+ *     CUDA device the device calls fail with ROCKET_ECUDA.
+ */
+#ifndef ROCKET_B200_H
+#define ROCKET_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rocket_params rocket_params_t; /* opaque: host arrays, device copies, launch plan */
+
+typedef enum {
+    ROCKET_OK = 0,
+    ROCKET_EINVAL = -1,       /* null pointer, negative size, parameter out of range            */
+    ROCKET_ESHAPE = -2,       /* C or L of the call differ from the handle's                    */
+    ROCKET_EUNSUPPORTED = -3, /* valid request outside what the kernels implement               */
+    ROCKET_ENOMEM = -4,       /* host or device allocation failed                               */
+    ROCKET_ECUDA = -5         /* a CUDA call failed (no device, launch error, copy error)       */
+} rocket_status_t;
+
+/* Largest kernel length and channel count per kernel the kernels are built for (Section 3.1
+ * draws lengths from {7, 9, 11} and at most min(C, len) channels). */
+#define ROCKET_MAX_LENGTH 11
+#define ROCKET_MAX_CHANNELS_PER_KERNEL 11
+
+/* Human-readable text for a status code.  Never NULL; static storage. */
+const char* rocket_strerror(int status);
+
+/*
+ * Random kernel initialisation (Section 3.1), on the host, from one seed.  Kernel k is a pure
+ * function of (seed, k, C, L): length uniform over {7,9,11}; weights N(0,1), each chosen
+ * channel's row mean-centred; bias U(-1,1); dilation floor(2^x), x ~ U(0, log2((L-1)/(len-1)));
+ * padding (len-1)d/2 with probability 1/2, else 0; floor(2^U(0, log2(min(C,len)+1))) channels
+ * drawn without replacement.  Draws are made in fp64 by a counter-based generator (splitmix64
+ * finaliser) and rounded once to fp32.  Needs K >= 1, C >= 1, L >= 11.  On success *out owns
+ * the host arrays and the launch plan; release with rocket_params_destroy.
+ */
+int rocket_params_generate(uint64_t seed, int K, int C, int L, rocket_params_t** out);
+
+/*
+ * Adopt caller-supplied kernels (the arrays are copied; the caller keeps ownership of its own).
+ * Requirements, else ROCKET_EINVAL: 1 <= length[k] <= 11; dilation[k] >= 1; padding[k] >= 0;
+ * L_out,k >= 1; 1 <= num_channels[k] <= min(C, 11); channel indices of one kernel distinct and
+ * in [0, C).  Any such kernel is accepted; lengths 7, 9 and 11 take the fast path.
+ */
+int rocket_params_from_arrays(int K, int C, int L, const int32_t* length, const int32_t* dilation,
+                              const int32_t* padding, const int32_t* num_channels,
+                              const int32_t* channel_idx, const float* weights, const float* bias,
+                              rocket_params_t** out);
+
+/* Sizes of the handle's arrays.  Any output pointer may be NULL. */
+int rocket_params_counts(const rocket_params_t* p, int* K, int* C, int* L, int64_t* n_channel_idx,
+                         int64_t* n_weights);
+
+/*
+ * Read-only views of the handle's host arrays (valid until rocket_params_destroy), so that a
+ * checker can consume exactly the numbers the device uses.  Any output pointer may be NULL.
+ */
+int rocket_params_host_view(const rocket_params_t* p, const int32_t** length, const int32_t** dilation,
+                            const int32_t** padding, const int32_t** num_channels,
+                            const int32_t** channel_idx, const float** weights, const float** bias);
+
+/* Convolution work of one example under the explicit count 2*len*channels*L_out summed over
+ * kernels (flop), and the number of conv outputs sum_k L_out,k.  Outputs may be NULL. */
+int rocket_params_work(const rocket_params_t* p, double* conv_flops_per_example,
+                       double* conv_outputs_per_example);
+
+/* Free the handle, its device copies and its workspace.  NULL is allowed.  The caller must
+ * have synchronised any stream that still runs work enqueued with this handle. */
+void rocket_params_destroy(rocket_params_t* p);
+
+/*
+ * Hard transform: PPV (Eq. 1-2, strict z > 0) and max for every (example, kernel).
+ *   X_dev    [N][C][L] fp32, device, 16-byte aligned;  C and L must equal the handle's
+ *   feat_dev [N][2K] fp32, device, written
+ * N = 0 is a successful no-op.
+ */
+int rocket_transform(const rocket_params_t* p, const float* X_dev, int N, int C, int L, float* feat_dev,
+                     void* cuda_stream);
+
+/*
+ * Soft transform: softPPV (Eq. 3-4) with softness lambda and shift (Eq. 3 as printed: shift =
+ * +3; the accompanying prose describes shift = -3; both are valid arguments), and max.
+ *   argmax_dev [N][K] int32, device, written when not NULL: the lowest output index attaining
+ *              the max, the sub-gradient choice the backward pass uses.
+ */
+int rocket_transform_soft(const rocket_params_t* p, const float* X_dev, int N, int C, int L, float lambda,
+                          float shift, float* feat_dev, int32_t* argmax_dev, void* cuda_stream);
+
+/*
+ * Backward of the soft transform for kernel weights and biases (the paper states that softPPV
+ * lets gradients flow; this is the chain rule through Eq. 3-4 and the convolution):
+ *   gz[n,k,i] = dfeat[n][2k] * (lambda / L_out) * h_i (1 - h_i) + dfeat[n][2k+1] * [i == argmax[n][k]]
+ *   db[k]       = sum_n sum_i gz[n,k,i]
+ *   dW_k[q][j]  = sum_n sum_i gz[n,k,i] * xpad[n, S_k[q], i - p_k + j d_k]
+ *   dfeat_dev  [N][2K] fp32, device      argmax_dev [N][K] int32, device (from the soft forward)
+ *   dW_dev     fp32, device, ragged exactly like the weights, assigned (not accumulated)
+ *   db_dev     [K] fp32, device, assigned
+ * No gradient with respect to X is produced.  N = 0 writes zeros.
+ */
+int rocket_transform_soft_backward(const rocket_params_t* p, const float* X_dev, int N, int C, int L,
+                                   float lambda, float shift, const float* dfeat_dev,
+                                   const int32_t* argmax_dev, float* dW_dev, float* db_dev,
+                                   void* cuda_stream);
+
+/*
+ * Host-buffer convenience forms of the three passes: inputs and outputs are HOST pointers
+ * (pinned memory makes the copies asynchronous, pageable memory works too).  The call copies the inputs to
+ * device buffers kept inside the handle (grown on demand, ROCKET_ENOMEM if that fails), runs
+ * the pass, copies the results back and returns after they have arrived.  argmax_host may be
+ * NULL in the forward; it is required in the backward.  These calls mutate the handle's
+ * staging buffers: one such call per handle at a time.
+ */
+int rocket_transform_host(rocket_params_t* p, const float* X_host, int N, int C, int L, float* feat_host);
+int rocket_transform_soft_host(rocket_params_t* p, const float* X_host, int N, int C, int L, float lambda,
+                               float shift, float* feat_host, int32_t* argmax_host);
+int rocket_transform_soft_backward_host(rocket_params_t* p, const float* X_host, int N, int C, int L,
+                                        float lambda, float shift, const float* dfeat_host,
+                                        const int32_t* argmax_host, float* dW_host, float* db_host);
+
+/*
+ * Which kernels serve the handle: 0 = automatic (fast path where it applies), 1 = force the
+ * generic kernels.  For tests and measurements; returns ROCKET_EINVAL for other values.
+ */
+int rocket_params_set_path(rocket_params_t* p, int path);
+
+/* Number of device kernels this library has launched in this process so far. */
+int64_t rocket_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ROCKET_B200_H */

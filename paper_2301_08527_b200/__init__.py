@@ -1,0 +1,11 @@
+"""B200-native ROCKET transform: thin Python binding over the C-ABI CUDA library.
+
+The binding only marshals arguments; every step of the transform runs in the CUDA kernels
+of librocket_b200.so.  There is no CPU fallback: importing works without a GPU (so the build
+can be checked), but every compute call needs a CUDA device and the compiled library.
+"""
+from .binding import (RocketError, RocketParams, kernel_launch_count, library_path, load_library,
+                      rocket_transform, rocket_transform_soft, rocket_transform_soft_backward)
+
+__all__ = ["RocketError", "RocketParams", "kernel_launch_count", "library_path", "load_library",
+           "rocket_transform", "rocket_transform_soft", "rocket_transform_soft_backward"]

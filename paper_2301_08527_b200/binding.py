@@ -1,0 +1,264 @@
+"""ctypes binding of include/rocket.h.  Same names as the C entry points; marshalling only.
+
+torch is used for device memory and streams; tensors are passed to the library as raw device
+pointers together with the current CUDA stream.
+"""
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "librocket_b200.so")
+_lib = None
+
+c_int32_p = ctypes.POINTER(ctypes.c_int32)
+c_float_p = ctypes.POINTER(ctypes.c_float)
+
+# name -> (restype, argtypes); every symbol include/rocket.h declares
+SIGNATURES = {
+    "rocket_strerror": (ctypes.c_char_p, [ctypes.c_int]),
+    "rocket_params_generate": (ctypes.c_int, [ctypes.c_uint64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                              ctypes.POINTER(ctypes.c_void_p)]),
+    "rocket_params_from_arrays": (ctypes.c_int, [ctypes.c_int, ctypes.c_int, ctypes.c_int] + [ctypes.c_void_p] * 7 +
+                                  [ctypes.POINTER(ctypes.c_void_p)]),
+    "rocket_params_counts": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int),
+                                            ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int64),
+                                            ctypes.POINTER(ctypes.c_int64)]),
+    "rocket_params_host_view": (ctypes.c_int, [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_void_p)] * 7),
+    "rocket_params_work": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_double),
+                                          ctypes.POINTER(ctypes.c_double)]),
+    "rocket_params_destroy": (None, [ctypes.c_void_p]),
+    "rocket_params_set_path": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
+    "rocket_kernel_launch_count": (ctypes.c_int64, []),
+    "rocket_transform": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                        ctypes.c_void_p, ctypes.c_void_p]),
+    "rocket_transform_soft": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                             ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_void_p,
+                                             ctypes.c_void_p, ctypes.c_void_p]),
+    "rocket_transform_soft_backward": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                                      ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_void_p,
+                                                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                                      ctypes.c_void_p]),
+    "rocket_transform_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                             ctypes.c_int, ctypes.c_void_p]),
+    "rocket_transform_soft_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                                  ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_void_p,
+                                                  ctypes.c_void_p]),
+    "rocket_transform_soft_backward_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                                                           ctypes.c_int, ctypes.c_int, ctypes.c_float, ctypes.c_float,
+                                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                                           ctypes.c_void_p]),
+}
+
+
+class RocketError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = int(status)
+        msg = load_library().rocket_strerror(self.status).decode()
+        super().__init__("%s failed: %s (status %d)" % (where, msg, self.status))
+
+
+def library_path():
+    return _LIB_PATH
+
+
+def load_library():
+    """Loads librocket_b200.so; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError("%s is missing: run `python -m paper_2301_08527_b200.build` "
+                               "(or __graft_entry__.build()) first; there is no CPU fallback" % _LIB_PATH)
+        lib = ctypes.CDLL(_LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def _check(status, where):
+    if status != 0:
+        raise RocketError(status, where)
+
+
+def kernel_launch_count():
+    return int(load_library().rocket_kernel_launch_count())
+
+
+def _np_ptr(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+class RocketParams:
+    """Owner of a rocket_params_t handle (kernel parameters on host and device)."""
+
+    def __init__(self, handle):
+        self._h = ctypes.c_void_p(handle)
+        lib = load_library()
+        K, C, L = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+        nch, nw = ctypes.c_int64(), ctypes.c_int64()
+        _check(lib.rocket_params_counts(self._h, K, C, L, nch, nw), "rocket_params_counts")
+        self.K, self.C, self.L = K.value, C.value, L.value
+        self.n_channel_idx, self.n_weights = nch.value, nw.value
+
+    @classmethod
+    def generate(cls, seed, K, C, L):
+        """rocket_params_generate: draw K kernels from one seed (Section 3.1)."""
+        h = ctypes.c_void_p()
+        _check(load_library().rocket_params_generate(ctypes.c_uint64(seed), K, C, L, ctypes.byref(h)),
+               "rocket_params_generate")
+        return cls(h.value)
+
+    @classmethod
+    def from_arrays(cls, K, C, L, length, dilation, padding, num_channels, channel_idx, weights, bias):
+        """rocket_params_from_arrays: adopt explicit kernels (numpy arrays are copied)."""
+        arrs = [np.ascontiguousarray(a, np.int32) for a in (length, dilation, padding, num_channels, channel_idx)]
+        arrs += [np.ascontiguousarray(a, np.float32) for a in (weights, bias)]
+        h = ctypes.c_void_p()
+        _check(load_library().rocket_params_from_arrays(K, C, L, *[_np_ptr(a) for a in arrs], ctypes.byref(h)),
+               "rocket_params_from_arrays")
+        return cls(h.value)
+
+    @classmethod
+    def from_kernel_params(cls, kp):
+        """Adopt any object with the fields of rocket_inputs.KernelParams."""
+        return cls.from_arrays(kp.K, kp.C, kp.L, kp.length, kp.dilation, kp.padding, kp.num_channels,
+                               kp.channel_idx, kp.weights, kp.bias)
+
+    def host_arrays(self):
+        """Copies of the handle's host arrays (rocket_params_host_view) as a dict of numpy arrays."""
+        ptrs = [ctypes.c_void_p() for _ in range(7)]
+        _check(load_library().rocket_params_host_view(self._h, *[ctypes.byref(p) for p in ptrs]),
+               "rocket_params_host_view")
+        names = ["length", "dilation", "padding", "num_channels", "channel_idx", "weights", "bias"]
+        sizes = [self.K, self.K, self.K, self.K, self.n_channel_idx, self.n_weights, self.K]
+        out = {}
+        for name, p, n in zip(names, ptrs, sizes):
+            ctype = ctypes.c_float if name in ("weights", "bias") else ctypes.c_int32
+            buf = (ctype * n).from_address(p.value) if n else (ctype * 0)()
+            out[name] = np.array(buf, copy=True)
+        return out
+
+    def work(self):
+        """(conv flop per example, conv outputs per example) under the count 2*len*channels*L_out."""
+        f, o = ctypes.c_double(), ctypes.c_double()
+        _check(load_library().rocket_params_work(self._h, f, o), "rocket_params_work")
+        return f.value, o.value
+
+    def set_path(self, path):
+        _check(load_library().rocket_params_set_path(self._h, int(path)), "rocket_params_set_path")
+
+    @property
+    def handle(self):
+        return self._h
+
+    def close(self):
+        if self._h is not None and self._h.value:
+            load_library().rocket_params_destroy(self._h)
+        self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def _dev_ptr(t, dtype, name):
+    import torch
+    if not isinstance(t, torch.Tensor) or not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError("%s must be a contiguous CUDA tensor of dtype %s" % (name, dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    import torch
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check_x(params, X):
+    if X.dim() != 3:
+        raise ValueError("X must be [N, C, L]")
+    return int(X.shape[0]), int(X.shape[1]), int(X.shape[2])
+
+
+def rocket_transform(params, X, out=None):
+    """Hard PPV + max.  X: CUDA fp32 [N, C, L] -> features CUDA fp32 [N, 2K] on the current stream."""
+    import torch
+    N, C, L = _check_x(params, X)
+    feat = out if out is not None else torch.empty((N, 2 * params.K), dtype=torch.float32, device=X.device)
+    _check(load_library().rocket_transform(params.handle, _dev_ptr(X, torch.float32, "X"), N, C, L,
+                                           _dev_ptr(feat, torch.float32, "out"), _stream()), "rocket_transform")
+    return feat
+
+
+def rocket_transform_soft(params, X, lam, shift=3.0, out=None, argmax_out=None, want_argmax=True):
+    """softPPV + max (Eq. 3-4).  Returns (features [N, 2K], argmax [N, K] int32 or None)."""
+    import torch
+    N, C, L = _check_x(params, X)
+    feat = out if out is not None else torch.empty((N, 2 * params.K), dtype=torch.float32, device=X.device)
+    arg = argmax_out
+    if arg is None and want_argmax:
+        arg = torch.empty((N, params.K), dtype=torch.int32, device=X.device)
+    _check(load_library().rocket_transform_soft(
+        params.handle, _dev_ptr(X, torch.float32, "X"), N, C, L, ctypes.c_float(lam), ctypes.c_float(shift),
+        _dev_ptr(feat, torch.float32, "out"),
+        _dev_ptr(arg, torch.int32, "argmax_out") if arg is not None else None, _stream()), "rocket_transform_soft")
+    return feat, arg
+
+
+def rocket_transform_soft_backward(params, X, lam, shift, dfeat, argmax, dW_out=None, db_out=None):
+    """Gradients of sum(dfeat * soft features) for weights (ragged like the weights) and biases."""
+    import torch
+    N, C, L = _check_x(params, X)
+    dW = dW_out if dW_out is not None else torch.empty((params.n_weights,), dtype=torch.float32, device=X.device)
+    db = db_out if db_out is not None else torch.empty((params.K,), dtype=torch.float32, device=X.device)
+    _check(load_library().rocket_transform_soft_backward(
+        params.handle, _dev_ptr(X, torch.float32, "X"), N, C, L, ctypes.c_float(lam), ctypes.c_float(shift),
+        _dev_ptr(dfeat, torch.float32, "dfeat"), _dev_ptr(argmax, torch.int32, "argmax"),
+        _dev_ptr(dW, torch.float32, "dW_out"), _dev_ptr(db, torch.float32, "db_out"), _stream()),
+        "rocket_transform_soft_backward")
+    return dW, db
+
+
+def _host_ptr(t, dtype, name):
+    import torch
+    if isinstance(t, np.ndarray):
+        t = torch.from_numpy(t)
+    if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError("%s must be a contiguous host tensor of dtype %s" % (name, dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def rocket_transform_host(params, X_host, feat_host):
+    """Host-buffer form: X_host / feat_host are host tensors (pinned for asynchronous copies)."""
+    import torch
+    N, C, L = _check_x(params, X_host)
+    _check(load_library().rocket_transform_host(params.handle, _host_ptr(X_host, torch.float32, "X_host"), N, C, L,
+                                                _host_ptr(feat_host, torch.float32, "feat_host")),
+           "rocket_transform_host")
+    return feat_host
+
+
+def rocket_transform_soft_host(params, X_host, lam, shift, feat_host, argmax_host=None):
+    import torch
+    N, C, L = _check_x(params, X_host)
+    _check(load_library().rocket_transform_soft_host(
+        params.handle, _host_ptr(X_host, torch.float32, "X_host"), N, C, L, ctypes.c_float(lam),
+        ctypes.c_float(shift), _host_ptr(feat_host, torch.float32, "feat_host"),
+        _host_ptr(argmax_host, torch.int32, "argmax_host") if argmax_host is not None else None),
+        "rocket_transform_soft_host")
+    return feat_host, argmax_host
+
+
+def rocket_transform_soft_backward_host(params, X_host, lam, shift, dfeat_host, argmax_host, dW_host, db_host):
+    import torch
+    N, C, L = _check_x(params, X_host)
+    _check(load_library().rocket_transform_soft_backward_host(
+        params.handle, _host_ptr(X_host, torch.float32, "X_host"), N, C, L, ctypes.c_float(lam),
+        ctypes.c_float(shift), _host_ptr(dfeat_host, torch.float32, "dfeat_host"),
+        _host_ptr(argmax_host, torch.int32, "argmax_host"), _host_ptr(dW_host, torch.float32, "dW_host"),
+        _host_ptr(db_host, torch.float32, "db_host")), "rocket_transform_soft_backward_host")
+    return dW_host, db_host

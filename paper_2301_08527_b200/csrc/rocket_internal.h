@@ -1,0 +1,53 @@
+// Internal declarations shared by the translation units of the ROCKET transform library.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+#include <vector>
+
+#include "rocket.h"
+
+namespace rocket {
+
+// Device-side view of the ragged kernel parameters (all pointers are device pointers).
+struct DeviceParams {
+    int K, C, L;
+    const int32_t* length;
+    const int32_t* dilation;
+    const int32_t* padding;
+    const int32_t* num_channels;
+    const int32_t* channel_offset;  // [K+1]
+    const int32_t* weight_offset;   // [K+1]
+    const int32_t* channel_idx;
+    const float* weights;
+    const float* bias;
+};
+
+struct HostParams {
+    int K = 0, C = 0, L = 0;
+    std::vector<int32_t> length, dilation, padding, num_channels, channel_idx;
+    std::vector<int32_t> channel_offset, weight_offset;  // [K+1]
+    std::vector<float> weights, bias;
+    double conv_flops = 0.0, conv_outputs = 0.0;
+};
+
+extern std::atomic<int64_t> g_launch_count;
+inline void count_launch(int n = 1) { g_launch_count.fetch_add(n, std::memory_order_relaxed); }
+
+// Draws K kernels by the rules of Section 3.1 with the counter-based generator.
+void generate_host_params(uint64_t seed, int K, int C, int L, HostParams& out);
+
+// ---- generic kernels (any length <= 11, any shape, no alignment demands) -------------------
+// Forward: one block per (example, kernel).  soft = false: PPV + max; soft = true: softPPV + max
+// (+ argmax when argmax != nullptr).
+cudaError_t launch_generic_forward(const DeviceParams& dp, const float* X, int N, bool soft, float lambda,
+                                   float shift, float* feat, int32_t* argmax, cudaStream_t stream);
+// Backward: per-example partial gradients into scratch[N][nW + K], then a fixed-order sum over n.
+size_t generic_backward_scratch_floats(int N, int64_t n_weights, int K);
+cudaError_t launch_generic_backward(const DeviceParams& dp, int64_t n_weights, const float* X, int N,
+                                    float lambda, float shift, const float* dfeat, const int32_t* argmax,
+                                    float* scratch, float* dW, float* db, cudaStream_t stream);
+
+}  // namespace rocket

@@ -8,10 +8,10 @@ the parameters of kernel k do not depend on K:
   slot 2   padding      (len-1)*d/2 when u < 0.5, else 0
   slot 3   channels     m = floor(2^(u * log2(min(C,len)+1))), clipped to [1, min(C,len)]
   slot 4   bias         2u - 1, uniform on [-1, 1)
-  slot 16+c            sort key of channel c; the m smallest keys are the chosen
-                       channels, listed in ascending channel order
   slot 64+2(11q+j), +1 Box-Muller pair for weight (q, j): sqrt(-2 ln u1) cos(2 pi u2),
                        u1 taken from (0, 1]
+  slot 1024+c          sort key of channel c; the m smallest keys are the chosen
+                       channels, listed in ascending channel order
 
 Weights are drawn in fp64, each chosen channel's row is mean-centred in fp64, and the
 result is rounded once to fp32.  Layout is ragged: kernel k owns num_channels[k]
@@ -26,8 +26,8 @@ from .rng import counter_u64, counter_uniform
 
 MAX_LEN = 11
 SLOT_LENGTH, SLOT_DILATION, SLOT_PADDING, SLOT_CHANNELS, SLOT_BIAS = 0, 1, 2, 3, 4
-SLOT_CHANNEL_KEYS = 16
 SLOT_WEIGHTS = 64
+SLOT_CHANNEL_KEYS = 1024
 
 
 @dataclass
