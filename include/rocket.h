@@ -100,6 +100,12 @@ int rocket_params_host_view(const rocket_params_t* p, const int32_t** length, co
 int rocket_params_work(const rocket_params_t* p, double* conv_flops_per_example,
                        double* conv_outputs_per_example);
 
+/*
+ * Bind the handle to the current CUDA device now (upload its parameters) instead of at its
+ * first device call.  Allocates device memory; a no-op returning ROCKET_OK when already bound.
+ */
+int rocket_params_bind_device(const rocket_params_t* p);
+
 /* Free the handle, its device copies and its workspace.  NULL is allowed.  The caller must
  * have synchronised any stream that still runs work enqueued with this handle. */
 void rocket_params_destroy(rocket_params_t* p);
@@ -161,6 +167,38 @@ int rocket_params_set_path(rocket_params_t* p, int path);
 
 /* Number of device kernels this library has launched in this process so far. */
 int64_t rocket_kernel_launch_count(void);
+
+/*
+ * Allocation-free form of rocket_transform_soft_backward.  (The paper has no counterpart; this
+ * entry point exists for callers that are not allowed to allocate device memory.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a real-time control loop
+ * that must not take the allocator's locks or its implicit device synchronisation, inside a
+ * host process whose memory pool is fixed at start-up, or on a stream that another component is
+ * recording.  rocket_transform_soft_backward keeps its per-example partial sums in a workspace
+ * that it grows with cudaMalloc on demand; this form keeps them in a fixed array that is part
+ * of the library image instead, so the call itself never allocates or frees anything.
+ *
+ * Same arguments, same results and same error rules as rocket_transform_soft_backward, plus:
+ *   - The scratch array holds ROCKET_NOALLOC_MAX_SCRATCH_FLOATS floats (16 MiB).  Every GPU
+ *     that loads the library carries it until the process exits.  The call needs
+ *     N * (n_weights + K) floats of it and returns ROCKET_EUNSUPPORTED, launching nothing,
+ *     when that is more than the array holds.
+ *   - The handle must already be bound to its device (rocket_params_bind_device, or any
+ *     earlier device call with it); binding allocates, so do it during set-up.  An unbound
+ *     handle gives ROCKET_EINVAL.
+ *   - The first call on each device looks up the array's device address (no allocation, but
+ *     a runtime query); make that first call during set-up, before any stream capture.
+ *   - All calls on one device share the one array, and it keeps the previous call's contents.
+ *     Nothing in it needs clearing: each call writes every element it later reads.  Two calls
+ *     that overlap on the GPU (different streams, no event between them) race on it and give
+ *     wrong gradients; order them on the device.
+ */
+#define ROCKET_NOALLOC_MAX_SCRATCH_FLOATS (4 * 1024 * 1024)
+int rocket_transform_soft_backward_noalloc(const rocket_params_t* p, const float* X_dev, int N, int C, int L,
+                                           float lambda, float shift, const float* dfeat_dev,
+                                           const int32_t* argmax_dev, float* dW_dev, float* db_dev,
+                                           void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -30,6 +30,11 @@ SIGNATURES = {
                                           ctypes.POINTER(ctypes.c_double)]),
     "rocket_params_destroy": (None, [ctypes.c_void_p]),
     "rocket_params_set_path": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
+    "rocket_params_bind_device": (ctypes.c_int, [ctypes.c_void_p]),
+    "rocket_transform_soft_backward_noalloc": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                                                              ctypes.c_int, ctypes.c_int, ctypes.c_float,
+                                                              ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p,
+                                                              ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "rocket_kernel_launch_count": (ctypes.c_int64, []),
     "rocket_transform": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                         ctypes.c_void_p, ctypes.c_void_p]),
@@ -147,6 +152,10 @@ class RocketParams:
         _check(load_library().rocket_params_work(self._h, f, o), "rocket_params_work")
         return f.value, o.value
 
+    def bind_device(self):
+        """rocket_params_bind_device: upload the parameters to the current device now."""
+        _check(load_library().rocket_params_bind_device(self._h), "rocket_params_bind_device")
+
     def set_path(self, path):
         _check(load_library().rocket_params_set_path(self._h, int(path)), "rocket_params_set_path")
 
@@ -221,6 +230,20 @@ def rocket_transform_soft_backward(params, X, lam, shift, dfeat, argmax, dW_out=
         _dev_ptr(dW, torch.float32, "dW_out"), _dev_ptr(db, torch.float32, "db_out"), _stream()),
         "rocket_transform_soft_backward")
     return dW, db
+
+
+def rocket_transform_soft_backward_noalloc(params, X, lam, shift, dfeat, argmax, dW_out, db_out):
+    """Allocation-free backward: same results as rocket_transform_soft_backward, scratch in a fixed
+    library-owned array (see include/rocket.h for its size limit and sharing rules).  The caller
+    supplies the outputs, and the handle must already be bound to the device."""
+    import torch
+    N, C, L = _check_x(params, X)
+    _check(load_library().rocket_transform_soft_backward_noalloc(
+        params.handle, _dev_ptr(X, torch.float32, "X"), N, C, L, ctypes.c_float(lam), ctypes.c_float(shift),
+        _dev_ptr(dfeat, torch.float32, "dfeat"), _dev_ptr(argmax, torch.int32, "argmax"),
+        _dev_ptr(dW_out, torch.float32, "dW_out"), _dev_ptr(db_out, torch.float32, "db_out"), _stream()),
+        "rocket_transform_soft_backward_noalloc")
+    return dW_out, db_out
 
 
 def _host_ptr(t, dtype, name):

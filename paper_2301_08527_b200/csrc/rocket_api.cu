@@ -1,7 +1,6 @@
 // C ABI of the ROCKET transform library: parameter handles, validation, dispatch.
 #include <algorithm>
 #include <cstring>
-#include <mutex>
 #include <new>
 
 #include "rocket_internal.h"
@@ -11,34 +10,6 @@ std::atomic<int64_t> g_launch_count{0};
 }
 
 using namespace rocket;
-
-// Grow-only device buffer owned by a handle.
-struct DeviceBuffer {
-    void* ptr = nullptr;
-    size_t bytes = 0;
-    cudaError_t reserve(size_t need) {
-        if (need <= bytes) return cudaSuccess;
-        if (ptr) cudaFree(ptr);
-        ptr = nullptr; bytes = 0;
-        cudaError_t e = cudaMalloc(&ptr, need);
-        if (e == cudaSuccess) bytes = need;
-        else ptr = nullptr;
-        return e;
-    }
-    void release() { if (ptr) cudaFree(ptr); ptr = nullptr; bytes = 0; }
-};
-
-struct rocket_params {
-    HostParams host;
-    int path = 0;                 // 0 = automatic, 1 = generic kernels only
-    mutable std::mutex mu;        // guards the lazy upload and the grow-only buffers below
-    mutable int device = -1;      // device of the first device call; -1 until then
-    mutable void* dev_blob = nullptr;  // one allocation holding every parameter array
-    mutable DeviceParams dp{};
-    mutable DeviceBuffer scratch; // backward partial sums
-    DeviceBuffer stage_x, stage_feat, stage_arg, stage_g, stage_dw;  // host-call staging
-    cudaStream_t host_stream = nullptr;
-};
 
 namespace {
 
@@ -264,6 +235,11 @@ void rocket_params_destroy(rocket_params_t* p) {
         cudaGetLastError();
     }
     delete p;
+}
+
+int rocket_params_bind_device(const rocket_params_t* p) {
+    if (!p) return ROCKET_EINVAL;
+    return ensure_device(p);
 }
 
 int rocket_params_set_path(rocket_params_t* p, int path) {

@@ -5,6 +5,7 @@
 
 #include <atomic>
 #include <cstdint>
+#include <mutex>
 #include <vector>
 
 #include "rocket.h"
@@ -51,3 +52,31 @@ cudaError_t launch_generic_backward(const DeviceParams& dp, int64_t n_weights, c
                                     float* scratch, float* dW, float* db, cudaStream_t stream);
 
 }  // namespace rocket
+
+// Grow-only device buffer owned by a handle.
+struct DeviceBuffer {
+    void* ptr = nullptr;
+    size_t bytes = 0;
+    cudaError_t reserve(size_t need) {
+        if (need <= bytes) return cudaSuccess;
+        if (ptr) cudaFree(ptr);
+        ptr = nullptr; bytes = 0;
+        cudaError_t e = cudaMalloc(&ptr, need);
+        if (e == cudaSuccess) bytes = need;
+        else ptr = nullptr;
+        return e;
+    }
+    void release() { if (ptr) cudaFree(ptr); ptr = nullptr; bytes = 0; }
+};
+
+struct rocket_params {
+    rocket::HostParams host;
+    int path = 0;                 // 0 = automatic, 1 = generic kernels only
+    mutable std::mutex mu;        // guards the lazy upload and the grow-only buffers below
+    mutable int device = -1;      // device of the first device call; -1 until then
+    mutable void* dev_blob = nullptr;  // one allocation holding every parameter array
+    mutable rocket::DeviceParams dp{};
+    mutable DeviceBuffer scratch; // backward partial sums
+    DeviceBuffer stage_x, stage_feat, stage_arg, stage_g, stage_dw;  // host-call staging
+    cudaStream_t host_stream = nullptr;
+};
