@@ -165,6 +165,14 @@ int rocket_transform_soft_backward_host(rocket_params_t* p, const float* X_host,
  */
 int rocket_params_set_path(rocket_params_t* p, int path);
 
+/*
+ * Device-side health of the handle.  Every wait inside the kernels (on a bulk-copy barrier) is
+ * bounded; a wait that gives up sets a flag instead of hanging the GPU, and the results of that
+ * call are then invalid.  This call synchronises the device, reads the flag into *wait_timeouts
+ * (0 = healthy) and returns ROCKET_OK unless the read itself failed.
+ */
+int rocket_params_device_status(const rocket_params_t* p, int* wait_timeouts);
+
 /* Number of device kernels this library has launched in this process so far. */
 int64_t rocket_kernel_launch_count(void);
 

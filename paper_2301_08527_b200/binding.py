@@ -31,6 +31,7 @@ SIGNATURES = {
     "rocket_params_destroy": (None, [ctypes.c_void_p]),
     "rocket_params_set_path": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
     "rocket_params_bind_device": (ctypes.c_int, [ctypes.c_void_p]),
+    "rocket_params_device_status": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int)]),
     "rocket_transform_soft_backward_noalloc": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
                                                               ctypes.c_int, ctypes.c_int, ctypes.c_float,
                                                               ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p,
@@ -155,6 +156,12 @@ class RocketParams:
     def bind_device(self):
         """rocket_params_bind_device: upload the parameters to the current device now."""
         _check(load_library().rocket_params_bind_device(self._h), "rocket_params_bind_device")
+
+    def device_status(self):
+        """rocket_params_device_status: number of bounded waits that gave up (0 = healthy)."""
+        flag = ctypes.c_int()
+        _check(load_library().rocket_params_device_status(self._h, flag), "rocket_params_device_status")
+        return flag.value
 
     def set_path(self, path):
         _check(load_library().rocket_params_set_path(self._h, int(path)), "rocket_params_set_path")

@@ -50,14 +50,16 @@ __device__ __forceinline__ float conv_at(const KernelShape& s, const float* __re
 template <bool SOFT>
 __global__ void __launch_bounds__(kThreads)
 generic_forward_kernel(DeviceParams dp, const float* __restrict__ X, float lambda, float shift,
-                       float* __restrict__ feat, int32_t* __restrict__ argmax) {
+                       float* __restrict__ feat, int32_t* __restrict__ argmax, const int32_t* __restrict__ klist,
+                       int nk) {
     __shared__ float sW[kMaxTaps];
     __shared__ int sS[ROCKET_MAX_CHANNELS_PER_KERNEL];
     __shared__ float rsum[kWarps], rmax[kWarps];
     __shared__ int rcnt[kWarps], rarg[kWarps];
 
     const int64_t e = blockIdx.x;
-    const int n = (int)(e / dp.K), k = (int)(e % dp.K);
+    const int n = (int)(e / nk);
+    const int k = klist ? klist[e % nk] : (int)(e % nk);
     const KernelShape s = load_kernel(dp, k, sW, sS);
     const float* Xn = X + (int64_t)n * dp.C * dp.L;
     const float b = dp.bias[k];
@@ -186,12 +188,14 @@ reduce_examples_kernel(const float* __restrict__ scratch, int N, int64_t n_weigh
 }  // namespace
 
 cudaError_t launch_generic_forward(const DeviceParams& dp, const float* X, int N, bool soft, float lambda,
-                                   float shift, float* feat, int32_t* argmax, cudaStream_t stream) {
-    const int64_t blocks = (int64_t)N * dp.K;
+                                   float shift, float* feat, int32_t* argmax, cudaStream_t stream,
+                                   const int32_t* klist, int nk) {
+    if (!klist) nk = dp.K;
+    const int64_t blocks = (int64_t)N * nk;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7fffffffll) return cudaErrorInvalidConfiguration;
-    if (soft) generic_forward_kernel<true><<<(unsigned)blocks, kThreads, 0, stream>>>(dp, X, lambda, shift, feat, argmax);
-    else generic_forward_kernel<false><<<(unsigned)blocks, kThreads, 0, stream>>>(dp, X, lambda, shift, feat, argmax);
+    if (soft) generic_forward_kernel<true><<<(unsigned)blocks, kThreads, 0, stream>>>(dp, X, lambda, shift, feat, argmax, klist, nk);
+    else generic_forward_kernel<false><<<(unsigned)blocks, kThreads, 0, stream>>>(dp, X, lambda, shift, feat, argmax, klist, nk);
     count_launch();
     return cudaGetLastError();
 }

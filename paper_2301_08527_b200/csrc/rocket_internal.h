@@ -42,9 +42,11 @@ void generate_host_params(uint64_t seed, int K, int C, int L, HostParams& out);
 
 // ---- generic kernels (any length <= 11, any shape, no alignment demands) -------------------
 // Forward: one block per (example, kernel).  soft = false: PPV + max; soft = true: softPPV + max
-// (+ argmax when argmax != nullptr).
+// (+ argmax when argmax != nullptr).  klist (device, nk entries) restricts the pass to those
+// kernels; nullptr means all K.
 cudaError_t launch_generic_forward(const DeviceParams& dp, const float* X, int N, bool soft, float lambda,
-                                   float shift, float* feat, int32_t* argmax, cudaStream_t stream);
+                                   float shift, float* feat, int32_t* argmax, cudaStream_t stream,
+                                   const int32_t* klist = nullptr, int nk = 0);
 // Backward: per-example partial gradients into scratch[N][nW + K], then a fixed-order sum over n.
 size_t generic_backward_scratch_floats(int N, int64_t n_weights, int K);
 cudaError_t launch_generic_backward(const DeviceParams& dp, int64_t n_weights, const float* X, int N,
@@ -52,6 +54,8 @@ cudaError_t launch_generic_backward(const DeviceParams& dp, int64_t n_weights, c
                                     float* scratch, float* dW, float* db, cudaStream_t stream);
 
 }  // namespace rocket
+
+namespace rocket { namespace fast { struct PlanHost; struct PlanDevice; } }
 
 // Grow-only device buffer owned by a handle.
 struct DeviceBuffer {
@@ -77,6 +81,9 @@ struct rocket_params {
     mutable void* dev_blob = nullptr;  // one allocation holding every parameter array
     mutable rocket::DeviceParams dp{};
     mutable DeviceBuffer scratch; // backward partial sums
+    rocket::fast::PlanHost* plan_host = nullptr;              // fast-path launch plan (host copy)
+    mutable rocket::fast::PlanDevice* plan_dev = nullptr;     // its device pointers, filled at binding
+    mutable void* plan_blob = nullptr;                        // one allocation holding the device plan
     DeviceBuffer stage_x, stage_feat, stage_arg, stage_g, stage_dw;  // host-call staging
     cudaStream_t host_stream = nullptr;
 };

@@ -30,6 +30,7 @@ def _run_hard(kp, X, path=0):
     p = rk.RocketParams.from_kernel_params(kp)
     p.set_path(path)
     feat = rk.rocket_transform(p, _dev(X)).cpu().numpy()
+    assert p.device_status() == 0
     p.close()
     return feat
 
