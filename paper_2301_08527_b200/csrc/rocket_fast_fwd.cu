@@ -139,28 +139,50 @@ __global__ void __launch_bounds__(kSThreads, 2) fast_s_forward(FwdArgs a) {
         const float* __restrict__ Xn = a.X + (size_t)n * a.C * a.L;
 
         // stage the tile: every channel, rows 0..rows-1 of every column, zero outside the series
-        const int nfill = a.C * b.rows;
-        for (int idx = warp; idx < nfill; idx += kSWarps) {
-            const int c = idx / b.rows, s = idx - c * b.rows;
+        for (int s = warp; s < b.rows; s += kSWarps) {
             const int xi = u0 + s * d;
-            float v = 0.0f;
-            if (lane_ok && xi >= 0 && xi < a.L) v = __ldg(Xn + (size_t)c * a.L + xi);
-            planes[(c * kRowsMax + s) * kSCols + lane] = v;
+            const bool ok = lane_ok && (unsigned)xi < (unsigned)a.L;
+            const float* __restrict__ src = Xn + (ok ? xi : 0);
+            float* dst = planes + s * kSCols + lane;
+#pragma unroll 4
+            for (int c = 0; c < a.C; ++c) {
+                float v = 0.0f;
+                if (ok) v = __ldg(src + (size_t)c * a.L);
+                dst[c * kSPlaneFloats] = v;
+            }
         }
         if (threadIdx.x == 0) s_next = b.kbeg;
         __syncthreads();
 
-        for (;;) {
-            int kk = 0;
-            if (lane == 0) kk = atomicAdd(&s_next, 1);
-            kk = __shfl_sync(kFull, kk, 0);
-            if (kk >= b.kend) break;
+        // kernels of the bucket, pulled from the shared counter; the parameters of the next kernel
+        // are fetched into registers while the current one computes
+        int kk = 0;
+        if (lane == 0) kk = atomicAdd(&s_next, 1);
+        kk = __shfl_sync(kFull, kk, 0);
+        int kb_next = 0;
+        float w_next[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+        auto prefetch = [&](int k) {
+            if (k < b.kend) {
+                kb_next = __ldg(reinterpret_cast<const int*>(a.plan.fk + k) + lane);
+                const float* wsrc = a.plan.negw + (size_t)k * kWeightsPerKernel;
+#pragma unroll
+                for (int i = 0; i < 5; ++i)
+                    if (lane + 32 * i < kWeightsPerKernel) w_next[i] = __ldg(wsrc + lane + 32 * i);
+            }
+        };
+        prefetch(kk);
+        while (kk < b.kend) {
             __syncwarp();
-            kb[lane] = __ldg(reinterpret_cast<const int*>(a.plan.fk + kk) + lane);
+            kb[lane] = kb_next;
+#pragma unroll
+            for (int i = 0; i < 5; ++i)
+                if (lane + 32 * i < kWeightsPerKernel) wb[lane + 32 * i] = w_next[i];
+            int kk_next = 0;
+            if (lane == 0) kk_next = atomicAdd(&s_next, 1);
+            kk_next = __shfl_sync(kFull, kk_next, 0);
+            prefetch(kk_next);
             __syncwarp();
-            const int len = kb[0], m = kb[3], woff = kb[5], korig = kb[6], lo_u = kb[7], hi_u = kb[8];
-            for (int i = lane; i < m * kWeightRow; i += 32) wb[i] = __ldg(a.plan.negw + woff + i);
-            __syncwarp();
+            const int len = kb[0], korig = kb[6], lo_u = kb[7], hi_u = kb[8];
             const bool mine = lane_ok && u0 >= lo_u && (u0 + (kBandRows - 1) * d) < hi_u;
             const bool interior = __all_sync(kFull, mine);
             int o_lo = 0, o_hi = kBandRows;
@@ -171,6 +193,7 @@ __global__ void __launch_bounds__(kSThreads, 2) fast_s_forward(FwdArgs a) {
             else if (len == 9) s_kernel_tile<9>(planes, wb, kb, lane, interior, o_lo, o_hi, cnt, mn);
             else s_kernel_tile<11>(planes, wb, kb, lane, interior, o_lo, o_hi, cnt, mn);
             publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
+            kk = kk_next;
         }
     }
 }

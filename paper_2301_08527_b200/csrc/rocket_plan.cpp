@@ -41,9 +41,11 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         f.negb = 0.0f - hp.bias[k];
         const int32_t* S = hp.channel_idx.data() + hp.channel_offset[k];
         const float* W = hp.weights.data() + hp.weight_offset[k];
+        // weights of fast kernel i live at negw[i * kWeightsPerKernel], rows padded to kWeightRow
+        out.negw.resize(out.negw.size() + kWeightsPerKernel, 0.0f);
         for (int q = 0; q < f.m; ++q) {
             f.ch[q] = S[q];
-            for (int j = 0; j < kWeightRow; ++j) out.negw.push_back(j < f.len ? 0.0f - W[q * f.len + j] : 0.0f);
+            for (int j = 0; j < f.len; ++j) out.negw[f.woff + q * kWeightRow + j] = 0.0f - W[q * f.len + j];
         }
         out.fk.push_back(f);
     };
