@@ -7,21 +7,17 @@
 // columns of A: output (t, r) needs A[t .. t+len-1][r].  A thread owns one column r and R
 // consecutive rows ("a band"), keeps R accumulators in registers and streams R+len-1 inputs
 // per channel past them, so every input is loaded once and used len times.  Lanes of a warp own
-// adjacent columns.
+// adjacent columns.  Columns of successive bands are strung together into one "raster"
+// (band-major, r-minor) and tiles are runs of consecutive raster positions, so lanes stay busy
+// even when d is smaller than a tile.
 //
 // Two regimes share the arithmetic core:
-//   S (d < split): kernels of one dilation form a bucket.  Columns of successive bands are
-//     strung together into one "raster" (band-major, r-minor) and a tile is 32 consecutive raster
-//     positions, so lanes stay busy even when d < 32.  A block stages one tile of ALL channels
-//     in shared memory (threads copy and zero-pad), then its warps pull kernels of the bucket
-//     from a shared counter, so one staged tile serves dozens to hundreds of kernels.
-//   T (d >= split): few kernels share a dilation, so a block takes one kernel, one band and 128
-//     adjacent residues, and streams the kernel's channels through a ring of shared-memory
-//     stages.  A producer warp fills the ring with tiled TMA loads: the zero-padded copy of the
-//     batch is viewed as a 2-D tensor with rows of 4d floats (row pitch 16d bytes, a legal TMA
-//     stride for every d), in which the rows s, s+4, s+8, .. of a tile's column block form one
-//     box; four boxes (one per s mod 4) bring a whole stage.  Consumer warps do nothing but
-//     shared-memory loads, FMAs and pooling.
+//   S (d < split): kernels of one dilation form a bucket; a block stages one 32-column tile of
+//     ALL channels in shared memory (threads copy and zero-pad), then its warps pull kernels of
+//     the bucket from a shared counter, so one staged tile serves dozens to hundreds of kernels.
+//   T (d >= split): few kernels share a dilation, so a block takes one kernel and a 128-column
+//     tile and streams the kernel's channels through a two-slot ring filled by bulk TMA row
+//     copies (no issue slots spent on the fill), overlapped with the FMAs of the previous channel.
 #pragma once
 
 #include <cstdint>
@@ -36,22 +32,17 @@ constexpr int kBandRows = 32;                                      // R of a ful
 constexpr int kWeightRow = 12;                                     // weights of one channel, padded
 constexpr int kWeightsPerKernel = kWeightRow * ROCKET_MAX_CHANNELS_PER_KERNEL;  // fixed stride in negw
 constexpr int kRowsMax = kBandRows + ROCKET_MAX_LENGTH - 1;        // staged rows per band
-constexpr int kSplitDefault = 72;                                  // S below, T at or above
+constexpr int kSplitDefault = 64;                                  // S below, T at or above
 constexpr int kSMaxChannels = 20;                                  // channels the S tile can stage
 
 constexpr int kSThreads = 256, kSWarps = kSThreads / 32, kSCols = 32;
 constexpr int kSPlaneFloats = kRowsMax * kSCols;                   // one channel of an S tile
 
-constexpr int kTConsumerWarps = 4, kTThreads = 32 * (kTConsumerWarps + 1), kTCols = 32 * kTConsumerWarps;
-constexpr int kTBoxCols = kTCols + 4;                              // 4 floats of 16-byte alignment slack
-constexpr int kTBoxRowsMax = (kRowsMax + 3) / 4;                   // rows of one phase (s mod 4)
-constexpr int kTPhaseFloats = (kTBoxCols * kTBoxRowsMax + 31) / 32 * 32;  // 128-byte aligned phases
-constexpr int kTStageFloats = 4 * kTPhaseFloats;
-constexpr int kTStages = 3;
-constexpr int kTParamBufs = kTStages + 1;
-// Smallest dilation of the T regime: with two tensor views whose bases differ by about 2d floats,
-// one of them always holds a 132-wide box without crossing the end of a 4d-wide tensor row.
-constexpr int kTMinDilation = 72;
+constexpr int kTThreads = 128, kTCols = 128, kTMaxChunks = 3;
+constexpr int kTPitch = 152;                                       // 128 + 3 * (3 + 4) rounded up to 8
+constexpr int kTStageFloats = kRowsMax * kTPitch;
+constexpr int kTStages = 2;
+constexpr int kZeroFloats = 256;                                   // zero page for out-of-range rows
 
 // One kernel as the fast kernels read it (32 words).
 struct alignas(16) FastKernel {
@@ -69,21 +60,10 @@ struct SBucket {
     int32_t kbeg, kend, rows, pad_;       // kernels [kbeg, kend) of fk; rows = 32 + max len - 1
 };
 struct SItem { int32_t bucket, c0; };
-
-// One T tile, with everything the producer warp needs (16 words).
-struct alignas(16) TItem {
-    int32_t fk, t0, R, r0;                // band starts at A-row t0, R rows, residues [r0, r0+128)
-    int32_t map, len, d, m;               // map: index of the tile's pair of tensor views
-    int32_t box_rows;                     // rows per phase box = ceil((R + len - 1) / 4)
-    uint8_t ch[12];
-    int32_t pad_[4];
+struct TItem {
+    int32_t fk, t0, R, c0;                // t0: A-row of band 0 of the item's band group
+    int32_t raster_len, pad_[3];
 };
-static_assert(sizeof(TItem) == 64, "TItem must be 16 words");
-struct TMapSpec { int32_t d, box_rows; };  // one pair of tensor views (bases 0 and ~2d floats)
-
-// Zero-padded copy of the batch the T regime reads: row (n, c) starts at float
-// front + (n*C + c) * pitch and is followed by at least `margin` zeros.
-struct PadLayout { int64_t front = 0, pitch = 0, margin = 0; };
 
 struct PlanHost {
     bool enabled = false;
@@ -93,9 +73,7 @@ struct PlanHost {
     std::vector<SBucket> sb;
     std::vector<SItem> sitems;
     std::vector<TItem> titems;
-    std::vector<TMapSpec> tspecs;
     std::vector<int32_t> generic_list;    // kernels the fast path does not take
-    PadLayout pad;
 };
 
 struct PlanDevice {
@@ -105,25 +83,16 @@ struct PlanDevice {
     const SItem* sitems = nullptr;
     const TItem* titems = nullptr;
     const int32_t* generic_list = nullptr;
+    const float* zeros = nullptr;
     unsigned* counters = nullptr;         // [0] S work counter, [1] T work counter
     int* error_flag = nullptr;            // set when a bounded wait gave up
-    const void* tmaps = nullptr;          // CUtensorMap[2 * n_tspecs], 128 bytes each
-    float* xpad = nullptr;                // zero-padded copy of the batch
-    int64_t pad_front = 0, pad_pitch = 0;
-    int n_fk = 0, n_sitems = 0, n_titems = 0, n_generic = 0, n_tspecs = 0;
+    int n_fk = 0, n_sitems = 0, n_titems = 0, n_generic = 0;
 };
 
 // Builds the launch plan for the kernels in hp (host side, once per handle).
 void build_plan(const HostParams& hp, int split, PlanHost& out);
 
-// Floats the padded copy needs for N examples.
-int64_t pad_buffer_floats(const PlanHost& plan, int N, int C);
-
-// Encodes the tensor views of every TMapSpec over a padded buffer of total_floats floats at
-// xpad (device address) into maps_host (2 * n_tspecs * 128 bytes).  Needs the CUDA driver.
-cudaError_t encode_tensor_maps(const PlanHost& plan, float* xpad, int64_t total_floats, void* maps_host);
-
-// Hard forward through the fast path: pad copy, init, S kernel, T kernel, finalise.
+// Hard forward through the fast path: init, S kernel, T kernel, finalise.  feat is [N][2K].
 cudaError_t launch_fast_forward(const PlanDevice& pd, const DeviceParams& dp, const float* X, int N, float* feat,
                                 cudaStream_t stream);
 

@@ -31,43 +31,67 @@ ROCKET_HD int s_column_u0(const SBucket& b, int cg) {
     return (b.tmin + band * kBandRows) * b.d + r;
 }
 
-// T regime.  Column lc (0..127) of a tile owns residue r0 + lc.  Row s of the tile (A-row t0 + s)
-// arrives with the box of phase s & 3; the box starts at a 16-byte aligned element, so the
-// wanted element sits `shift` floats into the box row, shift = (t0*d + r0 + (s & 3)*d) & 3
-// (rows 4 apart differ by 4d floats, which keeps the shift).
+// T regime: a tile is cut into chunks, runs of consecutive residues, one per band it touches.
+struct TChunk { int tb, ra, w, off; };  // first A-row, first residue, width, column offset in the stage row
+
+ROCKET_HD int t_make_chunks(const TItem& item, int d, TChunk (&chunks)[kTMaxChunks], int& ncols) {
+    const int band0 = item.c0 / d, rs = item.c0 - band0 * d;
+    ncols = imin(kTCols, item.raster_len - item.c0);
+    int remaining = ncols, ra = rs, band = band0, off = 0, nch = 0;
+    while (remaining > 0 && nch < kTMaxChunks) {
+        const int w = imin(d - ra, remaining);
+        chunks[nch].tb = item.t0 + band * item.R; chunks[nch].ra = ra; chunks[nch].w = w; chunks[nch].off = off;
+        off += ((w + 3) & ~3) + 4;
+        remaining -= w; ra = 0; ++band; ++nch;
+    }
+    return remaining > 0 ? -1 : nch;  // -1: the tile would need more chunks than the stage row holds
+}
+
+// Column lc of a T tile: its chunk, residue, first output's u, and the four shared-memory column
+// offsets (index = row & 3) that absorb the 16-byte alignment shift of each bulk-copied row.
 struct TColumn { int u0; int col[4]; bool ok; };
 
-ROCKET_HD TColumn t_column(int t0, int r0, int d, int lc) {
+ROCKET_HD TColumn t_column(const TChunk* chunks, int nch, int ncols, int d, int lc) {
     TColumn c;
-    c.ok = r0 + lc < d;
-    const int within = c.ok ? lc : 0;
-    c.u0 = t0 * d + r0 + within;
-    for (int j = 0; j < 4; ++j) c.col[j] = within + ((t0 * d + r0 + j * d) & 3);
+    c.ok = lc < ncols;
+    int start = 0, sel = 0;
+    for (int i = 0; i < nch; ++i) {
+        if (lc >= start && lc < start + chunks[i].w) sel = i;
+        start += chunks[i].w;
+    }
+    const TChunk ch = chunks[sel];
+    int within = lc;
+    for (int i = 0; i < sel; ++i) within -= chunks[i].w;
+    if (!c.ok) within = 0;
+    c.u0 = ch.tb * d + ch.ra + within;
+    for (int j = 0; j < 4; ++j) c.col[j] = ch.off + within + ((ch.tb * d + ch.ra + j * d) & 3);
     return c;
 }
 
-// Offset (floats) of row s inside a stage: phase block (s & 3), box row (s >> 2).
-ROCKET_HD constexpr int t_row_offset(int s) { return (s & 3) * kTPhaseFloats + (s >> 2) * kTBoxCols; }
+// One bulk copy of the fill: row s of chunk c.  Bytes [0, in_bytes) come from the series at
+// element offset src_elem of the channel row (or from the zero page when src_elem < 0), bytes
+// [in_bytes, tot_bytes) from the zero page.  dst_bytes is relative to the stage slot.
+struct TCopy { int src_elem; uint32_t dst_bytes, in_bytes, tot_bytes; };
 
-// One tiled TMA load of the fill: phase k of a stage.  e0 is the flat float index, in the padded
-// buffer, of the tile's row 0 / column 0 element for the stage's channel.  The buffer is seen
-// through one of two tensor views with rows of 4d floats: view 0 starts at float 0, view 1 at
-// float t_view_shift(d).  The box is kTBoxCols wide and starts at the 16-byte aligned coordinate
-// (x, y); the view is chosen so that the box does not cross the end of a tensor row.
-ROCKET_HD int t_view_shift(int d) { return (2 * d + 3) & ~3; }
-struct TBox { int view, x, y; };
-
-ROCKET_HD TBox t_box_of(uint32_t kappa0, uint32_t rho0, int k, int d) {
-    const uint32_t w = 4u * (uint32_t)d;
-    uint32_t kappa = kappa0 + (uint32_t)k * (uint32_t)d, rho = rho0;
-    if (kappa >= w) { kappa -= w; rho += 1; }
-    TBox b;
-    if ((kappa & ~3u) + (uint32_t)kTBoxCols <= w) {
-        b.view = 0; b.x = (int)(kappa & ~3u); b.y = (int)rho;
+ROCKET_HD TCopy t_copy_of(int task, const TChunk* chunks, int rows, int d, int L) {
+    const int c = task / rows, s = task - c * rows;
+    const TChunk ch = chunks[c];
+    const int t = ch.tb + s;
+    const int xs = t * d + ch.ra;
+    const int al = xs & 3;
+    TCopy cp;
+    cp.tot_bytes = (uint32_t)((al + ch.w + 3) & ~3) * 4u;
+    cp.dst_bytes = (uint32_t)(s * kTPitch + ch.off) * 4u;
+    if (t < 0 || xs >= L) {
+        cp.src_elem = -1; cp.in_bytes = cp.tot_bytes;
     } else {
-        b.view = 1; b.x = (int)((kappa - (uint32_t)t_view_shift(d)) & ~3u); b.y = (int)rho;
+        const int as = xs - al;
+        const int end = imin(xs + ch.w, L);
+        cp.src_elem = as;
+        const uint32_t in = (uint32_t)((end - as + 3) & ~3) * 4u;
+        cp.in_bytes = in < cp.tot_bytes ? in : cp.tot_bytes;
     }
-    return b;
+    return cp;
 }
 
 }  // namespace fast
