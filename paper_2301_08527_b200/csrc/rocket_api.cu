@@ -52,42 +52,6 @@ int validate_channels(const HostParams& hp) {
 
 size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
-// Uploads the fast-path plan (one allocation: kernels, weights, buckets, items, zero page,
-// work counters, error flag) and fills p->plan_dev.
-int upload_plan(const rocket_params* p) {
-    const fast::PlanHost& h = *p->plan_host;
-    fast::PlanDevice& d = *p->plan_dev;
-    d = fast::PlanDevice();
-    struct Part { const void* src; size_t bytes; size_t off; };
-    Part parts[9] = {
-        {h.fk.data(), h.fk.size() * sizeof(fast::FastKernel), 0}, {h.negw.data(), h.negw.size() * 4, 0},
-        {h.sb.data(), h.sb.size() * sizeof(fast::SBucket), 0},    {h.sitems.data(), h.sitems.size() * sizeof(fast::SItem), 0},
-        {h.titems.data(), h.titems.size() * sizeof(fast::TItem), 0},
-        {h.generic_list.data(), h.generic_list.size() * 4, 0},
-        {nullptr, fast::kZeroFloats * 4, 0}, {nullptr, 256, 0}, {nullptr, 256, 0}};
-    size_t total = 0;
-    for (auto& pt : parts) { pt.off = total; total += align256(pt.bytes); }
-    cudaError_t e = cudaMalloc(&p->plan_blob, std::max<size_t>(total, 256));
-    if (e != cudaSuccess) { cudaGetLastError(); p->plan_blob = nullptr; return e == cudaErrorMemoryAllocation ? ROCKET_ENOMEM : ROCKET_ECUDA; }
-    char* base = static_cast<char*>(p->plan_blob);
-    bool ok = cudaMemset(base, 0, std::max<size_t>(total, 256)) == cudaSuccess;
-    for (auto& pt : parts)
-        if (ok && pt.src && pt.bytes) ok = cudaMemcpy(base + pt.off, pt.src, pt.bytes, cudaMemcpyHostToDevice) == cudaSuccess;
-    if (!ok) { cudaGetLastError(); cudaFree(p->plan_blob); p->plan_blob = nullptr; return ROCKET_ECUDA; }
-    d.fk = reinterpret_cast<const fast::FastKernel*>(base + parts[0].off);
-    d.negw = reinterpret_cast<const float*>(base + parts[1].off);
-    d.sb = reinterpret_cast<const fast::SBucket*>(base + parts[2].off);
-    d.sitems = reinterpret_cast<const fast::SItem*>(base + parts[3].off);
-    d.titems = reinterpret_cast<const fast::TItem*>(base + parts[4].off);
-    d.generic_list = reinterpret_cast<const int32_t*>(base + parts[5].off);
-    d.zeros = reinterpret_cast<const float*>(base + parts[6].off);
-    d.counters = reinterpret_cast<unsigned*>(base + parts[7].off);
-    d.error_flag = reinterpret_cast<int*>(base + parts[8].off);
-    d.n_fk = (int)h.fk.size(); d.n_sitems = (int)h.sitems.size(); d.n_titems = (int)h.titems.size();
-    d.n_generic = (int)h.generic_list.size();
-    return ROCKET_OK;
-}
-
 // Uploads the host arrays into one device allocation on the current device and fills p->dp.
 // Runs once per handle, at its first device call.
 int ensure_device(const rocket_params* p) {
@@ -127,11 +91,14 @@ int ensure_device(const rocket_params* p) {
     d.channel_idx = reinterpret_cast<const int32_t*>(base + parts[6].off);
     d.weights = reinterpret_cast<const float*>(base + parts[7].off);
     d.bias = reinterpret_cast<const float*>(base + parts[8].off);
-    int st = upload_plan(p);
-    if (st != ROCKET_OK) {
-        cudaFree(p->dev_blob);
-        p->dev_blob = nullptr;
-        return st;
+    if (p->fast->host.enabled) {
+        cudaError_t pe = fast::upload_plan(*p->fast);
+        if (pe != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(p->dev_blob);
+            p->dev_blob = nullptr;
+            return pe == cudaErrorMemoryAllocation ? ROCKET_ENOMEM : ROCKET_ECUDA;
+        }
     }
     p->device = dev;
     return ROCKET_OK;
@@ -142,9 +109,8 @@ int finish_handle(rocket_params* p, rocket_params_t** out) {
     if (st == ROCKET_OK) st = validate_channels(p->host);
     if (st == ROCKET_OK) {
         try {
-            p->plan_host = new fast::PlanHost();
-            p->plan_dev = new fast::PlanDevice();
-            fast::build_plan(p->host, fast::kSplitDefault, *p->plan_host);
+            p->fast = new fast::FastState();
+            fast::build_plan(p->host, fast::kSplitDefault, p->fast->host);
         } catch (const std::bad_alloc&) {
             st = ROCKET_ENOMEM;
         }
@@ -280,15 +246,14 @@ void rocket_params_destroy(rocket_params_t* p) {
     if (p->device >= 0) {
         DeviceGuard g(p->device);
         if (p->dev_blob) cudaFree(p->dev_blob);
-        if (p->plan_blob) cudaFree(p->plan_blob);
+        if (p->fast) fast::release_fast_state(*p->fast);
         p->scratch.release();
         p->stage_x.release(); p->stage_feat.release(); p->stage_arg.release();
         p->stage_g.release(); p->stage_dw.release();
         if (p->host_stream) cudaStreamDestroy(p->host_stream);
         cudaGetLastError();
     }
-    delete p->plan_host;
-    delete p->plan_dev;
+    delete p->fast;
     delete p;
 }
 
@@ -300,10 +265,10 @@ int rocket_params_bind_device(const rocket_params_t* p) {
 int rocket_params_device_status(const rocket_params_t* p, int* wait_timeouts) {
     if (!p || !wait_timeouts) return ROCKET_EINVAL;
     *wait_timeouts = 0;
-    if (p->device < 0) return ROCKET_OK;
+    if (p->device < 0 || !p->fast->dev.error_flag) return ROCKET_OK;
     DeviceGuard g(p->device);
     if (!g.ok) return ROCKET_ECUDA;
-    return cuda_status(cudaMemcpy(wait_timeouts, p->plan_dev->error_flag, sizeof(int), cudaMemcpyDeviceToHost));
+    return cuda_status(cudaMemcpy(wait_timeouts, p->fast->dev.error_flag, sizeof(int), cudaMemcpyDeviceToHost));
 }
 
 int rocket_params_set_path(rocket_params_t* p, int path) {
@@ -325,12 +290,12 @@ int rocket_transform(const rocket_params_t* p, const float* X_dev, int N, int C,
     if (!g.ok) return ROCKET_ECUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const bool aligned = (reinterpret_cast<uintptr_t>(X_dev) & 15u) == 0;
-    if (p->path == 0 && p->plan_host->enabled && aligned) {
-        cudaError_t e = fast::launch_fast_forward(*p->plan_dev, p->dp, X_dev, N, feat_dev, stream);
+    if (p->path == 0 && p->fast->host.enabled && aligned) {
+        cudaError_t e = fast::launch_fast_forward(*p->fast, p->dp, X_dev, N, feat_dev, stream);
         if (e != cudaSuccess) return cuda_status(e);
-        if (p->plan_dev->n_generic == 0) return ROCKET_OK;
+        if (p->fast->dev.n_generic == 0) return ROCKET_OK;
         return cuda_status(launch_generic_forward(p->dp, X_dev, N, false, 0.0f, 0.0f, feat_dev, nullptr, stream,
-                                                  p->plan_dev->generic_list, p->plan_dev->n_generic));
+                                                  p->fast->dev.generic_list, p->fast->dev.n_generic));
     }
     return cuda_status(launch_generic_forward(p->dp, X_dev, N, false, 0.0f, 0.0f, feat_dev, nullptr, stream));
 }

@@ -4,20 +4,25 @@
 // Geometry.  A kernel with dilation d reads x[u + j*d] for output u = i - p (i the output
 // index, p the padding).  Writing u = t*d + r with 0 <= r < d turns the series into a 2-D array
 // A[t][r] = x[t*d + r], and the dilated convolution into a dense length-len filter down the
-// columns of A: output (t, r) needs A[t .. t+len-1][r].  A thread owns one column r and R
-// consecutive rows ("a band"), keeps R accumulators in registers and streams R+len-1 inputs
-// per channel past them, so every input is loaded once and used len times.  Lanes of a warp own
-// adjacent columns.  Columns of successive bands are strung together into one "raster"
-// (band-major, r-minor) and tiles are runs of consecutive raster positions, so lanes stay busy
-// even when d is smaller than a tile.
+// columns of A: output (t, r) needs A[t .. t+len-1][r].  A thread owns two adjacent columns
+// and 16 consecutive rows, keeps the 32 accumulators in registers as 16 packed pairs and
+// streams 16+len-1 input pairs per channel past them with packed two-wide FMAs
+// (fma.rn.f32x2), so every input is loaded once and used len times.  Lanes of a warp own
+// adjacent column pairs: a warp tile is 16 rows x 64 columns.
 //
 // Two regimes share the arithmetic core:
-//   S (d < split): kernels of one dilation form a bucket; a block stages one 32-column tile of
-//     ALL channels in shared memory (threads copy and zero-pad), then its warps pull kernels of
-//     the bucket from a shared counter, so one staged tile serves dozens to hundreds of kernels.
-//   T (d >= split): few kernels share a dilation, so a block takes one kernel and a 128-column
-//     tile and streams the kernel's channels through a two-slot ring filled by bulk TMA row
-//     copies (no issue slots spent on the fill), overlapped with the FMAs of the previous channel.
+//   S (d < split): kernels of one dilation form a bucket.  Columns of successive 16-row bands
+//     are strung together into one "raster" (band-major, r-minor) and a tile is 64 consecutive
+//     raster positions, so lanes stay busy even when d < 64.  A block stages one tile of ALL
+//     channels in shared memory, then its warps pull kernels of the bucket from a shared
+//     counter, so one staged tile serves dozens to hundreds of kernels.
+//   T (d >= split): few kernels share a dilation, so a block of four consumer warps takes one
+//     kernel and one tile (64 rows x 64 columns or 32 rows x 128 columns) and streams the
+//     kernel's channels through a ring of shared-memory stages.  A producer warp fills the
+//     ring with tiled TMA loads from a zero-margined copy of the batch, viewed as a 3-D tensor
+//     (x within a run of 4d floats, y = which run, z = channel row): rows s, s+4, s+8, .. of
+//     a tile are then one box, and four boxes (one per s mod 4) bring a whole stage without
+//     spending issue slots of the consumer warps.
 #pragma once
 
 #include <cstdint>
@@ -25,75 +30,123 @@
 
 #include "rocket_internal.h"
 
+#ifdef __CUDACC__
+#define ROCKET_CX __host__ __device__ constexpr
+#else
+#define ROCKET_CX constexpr
+#endif
+
 namespace rocket {
 namespace fast {
 
-constexpr int kBandRows = 32;                                      // R of a full band
-constexpr int kWeightRow = 12;                                     // weights of one channel, padded
-constexpr int kWeightsPerKernel = kWeightRow * ROCKET_MAX_CHANNELS_PER_KERNEL;  // fixed stride in negw
-constexpr int kRowsMax = kBandRows + ROCKET_MAX_LENGTH - 1;        // staged rows per band
+constexpr int kR = 16;                                             // output rows of a warp tile
+constexpr int kWarpCols = 64;                                      // columns of a warp tile (2 per lane)
+constexpr int kRowsMax = kR + ROCKET_MAX_LENGTH - 1;               // staged rows a warp tile reads
 constexpr int kSplitDefault = 64;                                  // S below, T at or above
-constexpr int kSMaxChannels = 20;                                  // channels the S tile can stage
+constexpr int kTMinDilation = 64;                                  // a T tile needs 64 residues in one band
 
-constexpr int kSThreads = 256, kSWarps = kSThreads / 32, kSCols = 32;
-constexpr int kSPlaneFloats = kRowsMax * kSCols;                   // one channel of an S tile
-
-constexpr int kTThreads = 128, kTCols = 128, kTMaxChunks = 3;
-constexpr int kTPitch = 152;                                       // 128 + 3 * (3 + 4) rounded up to 8
-constexpr int kTStageFloats = kRowsMax * kTPitch;
-constexpr int kTStages = 2;
-constexpr int kZeroFloats = 256;                                   // zero page for out-of-range rows
-
-// One kernel as the fast kernels read it (32 words).
-struct alignas(16) FastKernel {
+// ---- kernel record: one fast kernel as the device reads it (header + duplicated weights) ----
+constexpr int kPairRow = 24;                                       // floats of one channel's weight row
+struct alignas(16) KRec {
     int32_t len, d, p, m;
-    int32_t nout, woff, k, lo_u;   // woff: offset into negw; k: original kernel index; lo_u = -p
-    int32_t hi_u;                  // nout - p (exclusive bound on u)
+    int32_t nout, k, lo_u, hi_u;   // k: original kernel index; lo_u = -p; hi_u = nout - p (exclusive)
     float negb;                    // 0 - bias (never -0.0)
     int32_t ch[ROCKET_MAX_CHANNELS_PER_KERNEL];
-    int32_t pad_[11];
+    int32_t pad_[12];
+    // w2[q][2j] = w2[q][2j+1] = 0 - W[q][j]: each weight twice, ready as a packed pair
+    float w2[ROCKET_MAX_CHANNELS_PER_KERNEL][kPairRow];
 };
-static_assert(sizeof(FastKernel) == 128, "FastKernel must be 32 words");
+static_assert(sizeof(KRec) == 128 + 4 * ROCKET_MAX_CHANNELS_PER_KERNEL * kPairRow, "KRec layout");
+static_assert(sizeof(KRec) % 16 == 0, "KRec must be copyable in 16-byte pieces");
+
+// ---- S regime --------------------------------------------------------------------------------
+constexpr int kSMaxChannels = 20;                                  // channels the S tile can stage
+constexpr int kSThreads = 512, kSWarps = kSThreads / 32;
+constexpr int kSPlaneFloats = kRowsMax * kWarpCols;                // one channel of an S tile
 
 struct SBucket {
     int32_t d, tmin, nbands, raster_len;  // raster_len = nbands * d
-    int32_t kbeg, kend, rows, pad_;       // kernels [kbeg, kend) of fk; rows = 32 + max len - 1
+    int32_t kbeg, kend, rows, pad_;       // kernels [kbeg, kend) of krec; rows = 16 + max len - 1
 };
 struct SItem { int32_t bucket, c0; };
-struct TItem {
-    int32_t fk, t0, R, c0;                // t0: A-row of band 0 of the item's band group
-    int32_t raster_len, pad_[3];
+
+// ---- T regime --------------------------------------------------------------------------------
+constexpr int kTConsumerWarps = 4;
+constexpr int kTThreads = 32 * (kTConsumerWarps + 1);              // + one producer warp
+constexpr int kTBoxCols = kWarpCols + 4;                           // 4 floats of 16-byte alignment slack
+constexpr int kTStages = 2;
+constexpr int kTParamSlots = kTStages + 2;
+// Two tile shapes: shape 0 = 4 row groups x 1 column group (64 x 64 outputs),
+//                  shape 1 = 2 row groups x 2 column groups (32 x 128 outputs).
+ROCKET_CX int t_shape_rows(int shape) { return shape == 0 ? 64 : 32; }
+ROCKET_CX int t_shape_colgroups(int shape) { return shape == 0 ? 1 : 2; }
+// Box rows of one phase (rows s, s+4, ..), and the phase pitch in floats (a multiple of 32
+// floats keeps every box destination 128-byte aligned).
+ROCKET_CX int t_box_rows(int shape, int len) { return (t_shape_rows(shape) + len - 1 + 3) / 4; }
+ROCKET_CX int t_phase_floats(int box_rows) { return (box_rows * kTBoxCols + 31) / 32 * 32; }
+constexpr int kTStageFloats0 = 4 * t_phase_floats(t_box_rows(0, ROCKET_MAX_LENGTH));
+constexpr int kTStageFloats1 = 8 * t_phase_floats(t_box_rows(1, ROCKET_MAX_LENGTH));
+constexpr int kTStageFloats = kTStageFloats0 > kTStageFloats1 ? kTStageFloats0 : kTStageFloats1;
+constexpr int kTPadFront = 128;                                    // zero floats before every channel row
+constexpr int kTXExtra = 128;                                      // floats a box may run past a 4d run
+
+// One T tile with everything the producer warp needs (16 words).
+struct alignas(16) TItem {
+    int32_t tk, t0, r0, shape;            // tk: index into the T kernel list; tile origin (t0, r0)
+    int32_t d, len, m, box_rows;
+    uint8_t ch[12];
+    int32_t krec, pad_[4];                // krec: index into the kernel records
 };
+static_assert(sizeof(TItem) == 64, "TItem must be 16 words");
 
 struct PlanHost {
     bool enabled = false;
     int split = kSplitDefault;
-    std::vector<FastKernel> fk;
-    std::vector<float> negw;
+    std::vector<KRec> krec;
     std::vector<SBucket> sb;
     std::vector<SItem> sitems;
     std::vector<TItem> titems;
+    std::vector<int32_t> tkernels;        // krec index of every T kernel (tensor maps 2*i, 2*i+1 belong to it)
     std::vector<int32_t> generic_list;    // kernels the fast path does not take
+    int64_t pad_pitch = 0;                // floats per channel row of the zero-margined copy
 };
 
 struct PlanDevice {
-    const FastKernel* fk = nullptr;
-    const float* negw = nullptr;
+    const KRec* krec = nullptr;
     const SBucket* sb = nullptr;
     const SItem* sitems = nullptr;
     const TItem* titems = nullptr;
     const int32_t* generic_list = nullptr;
-    const float* zeros = nullptr;
-    unsigned* counters = nullptr;         // [0] S work counter, [1] T work counter
+    unsigned* counters = nullptr;         // [0] S work counter
     int* error_flag = nullptr;            // set when a bounded wait gave up
-    int n_fk = 0, n_sitems = 0, n_titems = 0, n_generic = 0;
+    const void* tmaps = nullptr;          // CUtensorMap[2 * n_tkernels], 128 bytes each
+    float* xpad = nullptr;                // zero-margined copy of the batch
+    int64_t pad_pitch = 0;
+    int n_krec = 0, n_sitems = 0, n_titems = 0, n_generic = 0, n_tkernels = 0;
 };
 
 // Builds the launch plan for the kernels in hp (host side, once per handle).
 void build_plan(const HostParams& hp, int split, PlanHost& out);
 
-// Hard forward through the fast path: init, S kernel, T kernel, finalise.  feat is [N][2K].
-cudaError_t launch_fast_forward(const PlanDevice& pd, const DeviceParams& dp, const float* X, int N, float* feat,
+// Device-side state of the fast path owned by a handle.
+struct FastState {
+    PlanHost host;
+    PlanDevice dev;
+    void* plan_blob = nullptr;            // records, buckets, items, counters, error flag
+    void* maps_blob = nullptr;            // tensor maps
+    float* xpad = nullptr;                // padded copy, capacity pad_examples
+    int pad_examples = 0;
+};
+
+// Uploads the plan (once per handle, at binding).
+cudaError_t upload_plan(FastState& fs);
+// Frees everything upload_plan / ensure_pad_capacity allocated.
+void release_fast_state(FastState& fs);
+// Makes the padded copy hold N examples and (re-)encodes the tensor maps over it.
+cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L);
+
+// Hard forward through the fast path: pad copy, init, S kernel, T kernel, finalise.
+cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const float* X, int N, float* feat,
                                 cudaStream_t stream);
 
 }  // namespace fast

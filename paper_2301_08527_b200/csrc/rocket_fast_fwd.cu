@@ -4,15 +4,21 @@
 //   - Accumulators hold -z: weights and bias are stored negated (acc = (0 - b) + sum (-w) x).  Then
 //     z > 0  <=>  the sign bit of acc is set, exactly: a zero accumulator is always +0 (it starts
 //     at +0 when b == 0, exact cancellation rounds to +0, and +0 plus a -0 product stays +0), so
-//     the PPV count is one shift-and-add per output and MAX = -min(acc) one min per output.
+//     the PPV count is one shift-and-add per output and MAX = -min(acc).
+//   - A thread's two columns travel together as one packed pair (fma.rn.f32x2 gives each half the
+//     result of a separate fused multiply-add).
 //   - Outputs outside the kernel's range are replaced by +inf before pooling (sign bit clear,
 //     neutral for the min).
 //   - Per (example, kernel) the count is combined with integer atomic adds and the max with an
 //     integer atomic max on an order-preserving key, both exact and order-independent, so the
 //     result is run-to-run identical.  The feature buffer itself holds these integers until the
 //     finalise kernel turns them into (count / L_out, max).
+#include <cuda.h>
+
+#include <algorithm>
 #include <cfloat>
 #include <climits>
+#include <cstring>
 
 #include "rocket_fast.h"
 #include "rocket_fast_geom.h"
@@ -21,9 +27,28 @@ namespace rocket {
 namespace fast {
 namespace {
 
+typedef unsigned long long u64;
 constexpr unsigned kFull = 0xffffffffu;
+constexpr long long kWaitLimitClocks = 1ll << 31;  // about a second: no wait inside a kernel lasts longer
 
-extern __shared__ __align__(128) float smem[];
+extern __shared__ __align__(128) unsigned char smem_raw[];
+
+__device__ __forceinline__ u64 pack2(float lo, float hi) {
+    u64 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void fma2(u64& acc, u64 a, u64 b) {
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 
 // Order-preserving map float -> signed int (for atomicMax) and back.
 __device__ __forceinline__ int float_key(float v) {
@@ -32,46 +57,55 @@ __device__ __forceinline__ int float_key(float v) {
 }
 __device__ __forceinline__ float key_float(int k) { return __int_as_float(k >= 0 ? k : k ^ 0x7fffffff); }
 
-// One channel of one band: R outputs down a column, R+ELL-1 inputs streamed past them.
-// Row s of the column sits at sm[col[s & 3] + s * PITCH]; the four column offsets absorb the
-// per-row 16-byte alignment shift of bulk-copied rows (all four are equal in the S regime).
-template <int ELL, int R, int PITCH>
-__device__ __forceinline__ void conv_channel(const float* __restrict__ sm, const int (&col)[4],
-                                             const float* __restrict__ w, float (&acc)[R]) {
-    const float4 w0 = *reinterpret_cast<const float4*>(w);
-    const float4 w1 = *reinterpret_cast<const float4*>(w + 4);
-    const float4 w2 = *reinterpret_cast<const float4*>(w + 8);
-    const float wall[12] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w, w2.x, w2.y, w2.z, w2.w};
-    float wr[ELL];
+// One channel of one warp tile: 16 output rows of the thread's column pair, 16+ELL-1 input pairs
+// streamed past them.  Row s of the tile sits at st[off[s & 3] + (s >> 2) * STEP]; w2 holds the
+// channel's negated weights, each twice.  With ODD, rows of odd s are only 4-byte aligned.
+template <int ELL, bool ODD, int STEP>
+__device__ __forceinline__ void conv_channel(const float* __restrict__ st, const int (&off)[4],
+                                             const float* __restrict__ w2, u64 (&acc)[kR]) {
+    u64 wp[ELL + 1];
 #pragma unroll
-    for (int j = 0; j < ELL; ++j) wr[j] = wall[j];
+    for (int j = 0; j < ELL; j += 2) {
+        const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(w2 + 2 * j);
+        wp[j] = v.x;
+        wp[j + 1] = v.y;
+    }
 #pragma unroll
-    for (int s = 0; s < R + ELL - 1; ++s) {
-        const float x = sm[col[s & 3] + s * PITCH];
+    for (int s = 0; s < kR + ELL - 1; ++s) {
+        const float* p = st + off[s & 3] + (s >> 2) * STEP;
+        u64 x;
+        if (ODD && (s & 1)) x = pack2(p[0], p[1]);
+        else x = *reinterpret_cast<const u64*>(p);
 #pragma unroll
         for (int j = 0; j < ELL; ++j) {
             const int o = s - j;
-            if (o >= 0 && o < R) acc[o] = fmaf(wr[j], x, acc[o]);
+            if (o >= 0 && o < kR) fma2(acc[o], wp[j], x);
         }
     }
 }
 
-// PPV count and min(-z) over the thread's R outputs; rows outside [o_lo, o_hi) are neutralised.
-template <int R>
-__device__ __forceinline__ void pool_hard(const float (&acc)[R], bool interior, int o_lo, int o_hi, int& cnt,
-                                          float& mn) {
+// PPV count and min(-z) over the thread's 2 x 16 outputs; rows outside [lo, hi) of either column
+// are neutralised.
+__device__ __forceinline__ void pool_hard(const u64 (&acc)[kR], bool interior, int lo0, int hi0, int lo1, int hi1,
+                                          int& cnt, float& mn) {
+    const float inf = __int_as_float(0x7f800000);
     if (interior) {
 #pragma unroll
-        for (int o = 0; o < R; ++o) {
-            cnt += (int)(__float_as_uint(acc[o]) >> 31);
-            mn = fminf(mn, acc[o]);
+        for (int o = 0; o < kR; ++o) {
+            float a, b;
+            unpack2(acc[o], a, b);
+            cnt += (int)(__float_as_uint(a) >> 31) + (int)(__float_as_uint(b) >> 31);
+            mn = min3(mn, a, b);
         }
     } else {
 #pragma unroll
-        for (int o = 0; o < R; ++o) {
-            const float a = (o >= o_lo && o < o_hi) ? acc[o] : __int_as_float(0x7f800000);
-            cnt += (int)(__float_as_uint(a) >> 31);
-            mn = fminf(mn, a);
+        for (int o = 0; o < kR; ++o) {
+            float a, b;
+            unpack2(acc[o], a, b);
+            if (o < lo0 || o >= hi0) a = inf;
+            if (o < lo1 || o >= hi1) b = inf;
+            cnt += (int)(__float_as_uint(a) >> 31) + (int)(__float_as_uint(b) >> 31);
+            mn = min3(mn, a, b);
         }
     }
 }
@@ -85,6 +119,8 @@ __device__ __forceinline__ void publish(int* __restrict__ feat_i, int64_t pair, 
     }
 }
 
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
 struct FwdArgs {
     PlanDevice plan;
     const float* X;
@@ -95,33 +131,36 @@ struct FwdArgs {
 // ------------------------------------------------------------------------------------------------
 // S regime
 // ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void cp_async4_zfill(uint32_t dst, const void* src, bool ok) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(ok ? 4 : 0) : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 template <int ELL>
-__device__ __forceinline__ void s_kernel_tile(const float* planes, const float* wb, const int* kb, int lane,
-                                              bool interior, int o_lo, int o_hi, int& cnt, float& mn) {
-    float acc[kBandRows];
-    const float negb = __int_as_float(kb[9]);
+__device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* rec, int lane, u64 (&acc)[kR]) {
+    const u64 negb = pack2(rec->negb, rec->negb);
 #pragma unroll
-    for (int o = 0; o < kBandRows; ++o) acc[o] = negb;
-    const int m = kb[3];
-    for (int q = 0; q < m; ++q) {
-        const int base = kb[10 + q] * kSPlaneFloats + lane;
-        const int col[4] = {base, base, base, base};
-        conv_channel<ELL, kBandRows, kSCols>(planes, col, wb + q * kWeightRow, acc);
-    }
-    pool_hard<kBandRows>(acc, interior, o_lo, o_hi, cnt, mn);
+    for (int o = 0; o < kR; ++o) acc[o] = negb;
+    const int m = rec->m;
+    const int off[4] = {2 * lane, kWarpCols + 2 * lane, 2 * kWarpCols + 2 * lane, 3 * kWarpCols + 2 * lane};
+    for (int q = 0; q < m; ++q)
+        conv_channel<ELL, false, 4 * kWarpCols>(planes + rec->ch[q] * kSPlaneFloats, off, rec->w2[q], acc);
 }
 
-__global__ void __launch_bounds__(kSThreads, 2) fast_s_forward(FwdArgs a) {
-    float* planes = smem;                                        // [C][kRowsMax][32]
-    float* wbuf = planes + a.C * kSPlaneFloats;                  // [warps][11 * 12]
-    int* kbuf = reinterpret_cast<int*>(wbuf + kSWarps * ROCKET_MAX_CHANNELS_PER_KERNEL * kWeightRow);  // [warps][32]
+__global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
+    float* planes = reinterpret_cast<float*>(smem_raw);                               // [C][kRowsMax][64]
+    KRec* recs = reinterpret_cast<KRec*>(planes + a.C * kSPlaneFloats);                // [warps][2]
     __shared__ unsigned s_item;
     __shared__ int s_next;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const unsigned n_items = (unsigned)a.plan.n_sitems;
     const unsigned long long total = (unsigned long long)a.N * n_items;
-    float* wb = wbuf + warp * (ROCKET_MAX_CHANNELS_PER_KERNEL * kWeightRow);
-    int* kb = kbuf + warp * 32;
+    KRec* myrec = recs + warp * 2;
 
     for (;;) {
         __syncthreads();  // the previous tile is fully consumed
@@ -133,256 +172,442 @@ __global__ void __launch_bounds__(kSThreads, 2) fast_s_forward(FwdArgs a) {
         const SItem item = a.plan.sitems[g - (unsigned)n * n_items];
         const SBucket b = a.plan.sb[item.bucket];
         const int d = b.d;
-        const int cg = item.c0 + lane;
-        const bool lane_ok = cg < b.raster_len;
-        const int u0 = s_column_u0(b, cg);  // u of the thread's first output row
         const float* __restrict__ Xn = a.X + (size_t)n * a.C * a.L;
 
         // stage the tile: every channel, rows 0..rows-1 of every column, zero outside the series
-        for (int s = warp; s < b.rows; s += kSWarps) {
-            const int xi = u0 + s * d;
-            const bool ok = lane_ok && (unsigned)xi < (unsigned)a.L;
-            const float* __restrict__ src = Xn + (ok ? xi : 0);
-            float* dst = planes + s * kSCols + lane;
+        {
+            const int col = threadIdx.x & (kWarpCols - 1), rg = threadIdx.x / kWarpCols;
+            const int cg = item.c0 + col;
+            const bool col_ok = cg < b.raster_len;
+            const int fu0 = s_column_u0(b, cg);
+            for (int s = rg; s < b.rows; s += kSThreads / kWarpCols) {
+                const int xi = fu0 + s * d;
+                const bool ok = col_ok && (unsigned)xi < (unsigned)a.L;
+                const float* __restrict__ src = Xn + (ok ? xi : 0);
+                uint32_t dst = smem_u32(planes + s * kWarpCols + col);
 #pragma unroll 4
-            for (int c = 0; c < a.C; ++c) {
-                float v = 0.0f;
-                if (ok) v = __ldg(src + (size_t)c * a.L);
-                dst[c * kSPlaneFloats] = v;
+                for (int c = 0; c < a.C; ++c) {
+                    cp_async4_zfill(dst, src, ok);
+                    src += a.L;
+                    dst += kSPlaneFloats * 4;
+                }
             }
+            cp_async_commit();
         }
+        // the thread's two columns
+        const int cg0 = item.c0 + 2 * lane;
+        const bool ok0 = cg0 < b.raster_len, ok1 = cg0 + 1 < b.raster_len;
+        const int u00 = s_column_u0(b, cg0), u01 = s_column_u0(b, cg0 + 1);
         if (threadIdx.x == 0) s_next = b.kbeg;
+        cp_async_wait<0>();
         __syncthreads();
 
-        // kernels of the bucket, pulled from the shared counter; the parameters of the next kernel
-        // are fetched into registers while the current one computes
+        // kernels of the bucket, pulled from the shared counter; the record of the next kernel is
+        // copied into the warp's other slot while the current one computes
+        auto fetch = [&](int k, int slot) {
+            if (k < b.kend) {
+                const char* src = reinterpret_cast<const char*>(a.plan.krec + k);
+                const uint32_t dst = smem_u32(myrec + slot);
+                for (int i = lane; i < (int)(sizeof(KRec) / 16); i += 32) cp_async16(dst + 16 * i, src + 16 * i);
+            }
+            cp_async_commit();
+        };
         int kk = 0;
         if (lane == 0) kk = atomicAdd(&s_next, 1);
         kk = __shfl_sync(kFull, kk, 0);
-        int kb_next = 0;
-        float w_next[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
-        auto prefetch = [&](int k) {
-            if (k < b.kend) {
-                kb_next = __ldg(reinterpret_cast<const int*>(a.plan.fk + k) + lane);
-                const float* wsrc = a.plan.negw + (size_t)k * kWeightsPerKernel;
-#pragma unroll
-                for (int i = 0; i < 5; ++i)
-                    if (lane + 32 * i < kWeightsPerKernel) w_next[i] = __ldg(wsrc + lane + 32 * i);
-            }
-        };
-        prefetch(kk);
+        int cur = 0;
+        fetch(kk, cur);
         while (kk < b.kend) {
-            __syncwarp();
-            kb[lane] = kb_next;
-#pragma unroll
-            for (int i = 0; i < 5; ++i)
-                if (lane + 32 * i < kWeightsPerKernel) wb[lane + 32 * i] = w_next[i];
             int kk_next = 0;
             if (lane == 0) kk_next = atomicAdd(&s_next, 1);
             kk_next = __shfl_sync(kFull, kk_next, 0);
-            prefetch(kk_next);
+            fetch(kk_next, cur ^ 1);
+            cp_async_wait<1>();
             __syncwarp();
-            const int len = kb[0], korig = kb[6], lo_u = kb[7], hi_u = kb[8];
-            const bool mine = lane_ok && u0 >= lo_u && (u0 + (kBandRows - 1) * d) < hi_u;
+            const KRec* rec = myrec + cur;
+            const int len = rec->len, korig = rec->k, lo_u = rec->lo_u, hi_u = rec->hi_u;
+            const bool mine = ok0 && ok1 && u00 >= lo_u && u01 >= lo_u && (u00 + (kR - 1) * d) < hi_u &&
+                              (u01 + (kR - 1) * d) < hi_u;
             const bool interior = __all_sync(kFull, mine);
-            int o_lo = 0, o_hi = kBandRows;
-            if (!interior) valid_rows(u0, d, lo_u, hi_u, kBandRows, lane_ok, o_lo, o_hi);
+            int lo0 = 0, hi0 = kR, lo1 = 0, hi1 = kR;
+            if (!interior) {
+                valid_rows(u00, d, lo_u, hi_u, kR, ok0, lo0, hi0);
+                valid_rows(u01, d, lo_u, hi_u, kR, ok1, lo1, hi1);
+            }
+            u64 acc[kR];
+            if (len == 7) s_kernel_tile<7>(planes, rec, lane, acc);
+            else if (len == 9) s_kernel_tile<9>(planes, rec, lane, acc);
+            else s_kernel_tile<11>(planes, rec, lane, acc);
             int cnt = 0;
             float mn = __int_as_float(0x7f800000);
-            if (len == 7) s_kernel_tile<7>(planes, wb, kb, lane, interior, o_lo, o_hi, cnt, mn);
-            else if (len == 9) s_kernel_tile<9>(planes, wb, kb, lane, interior, o_lo, o_hi, cnt, mn);
-            else s_kernel_tile<11>(planes, wb, kb, lane, interior, o_lo, o_hi, cnt, mn);
+            pool_hard(acc, interior, lo0, hi0, lo1, hi1, cnt, mn);
             publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
+            __syncwarp();  // every lane is done with the record before its slot is refilled
             kk = kk_next;
+            cur ^= 1;
         }
+        cp_async_wait<0>();
     }
 }
 
 // ------------------------------------------------------------------------------------------------
 // T regime
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait on a phase parity: returns false when the limit is reached (the caller records it).
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+// Wait on a phase parity, bounded in time: returns false when the limit is reached (the caller
+// records it and the block winds down).  Between polls the warp sleeps, so a waiting warp does
+// not take issue slots from the warps that compute.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (int it = 0; it < (1 << 20); ++it) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return true;
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        __nanosleep(64);
+        if (mbar_try(bar, parity)) return true;
+        if (clock64() - t0 > kWaitLimitClocks) return false;
     }
-    return false;
 }
 // Bulk copy global -> shared (16-byte aligned addresses, size a multiple of 16), completion on bar.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-
-// Warp 0 fills one ring slot with one channel of the tile: one bulk copy per (chunk, row), the
-// source rounded down to 16 bytes; rows or tails outside the series come from the zero page.
-__device__ __noinline__ void t_issue_stage(const float* __restrict__ xrow, const float* __restrict__ zeros,
-                                           const TChunk* chunks, int nch, int rows, int d, int L, uint32_t stage,
-                                           uint32_t bar, int lane) {
-    const int tasks = nch * rows;
-    uint32_t mine = 0;
-    for (int task = lane; task < tasks; task += 32) mine += t_copy_of(task, chunks, rows, d, L).tot_bytes;
-    const uint32_t total = __reduce_add_sync(kFull, mine);
-    if (lane == 0) mbar_arrive_expect_tx(bar, total);
-    __syncwarp();
-    for (int task = lane; task < tasks; task += 32) {
-        const TCopy cp = t_copy_of(task, chunks, rows, d, L);
-        const uint32_t dst = stage + cp.dst_bytes;
-        bulk_g2s(dst, cp.src_elem >= 0 ? xrow + cp.src_elem : zeros, cp.in_bytes, bar);
-        if (cp.in_bytes < cp.tot_bytes) bulk_g2s(dst + cp.in_bytes, zeros, cp.tot_bytes - cp.in_bytes, bar);
-    }
+// Tiled TMA load of one 3-D box (x a multiple of 4 floats), completion on bar.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
 
-template <int ELL, int R>
-__device__ __forceinline__ void t_kernel_tile(const FwdArgs& a, const float* stages, const float* wbuf,
-                                              const int* kb, const TChunk* chunks, int nch, const float* Xn,
-                                              const int (&col)[4], uint32_t bar0, uint32_t (&phase)[kTStages],
-                                              bool interior, int o_lo, int o_hi, int& cnt, float& mn) {
-    float acc[R];
-    const float negb = __int_as_float(kb[9]);
-#pragma unroll
-    for (int o = 0; o < R; ++o) acc[o] = negb;
-    const int m = kb[3], d = kb[1];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr int rows = R + ELL - 1;
+struct TParams {
+    KRec rec;
+    TItem item;
+};
+static_assert(sizeof(TParams) % 16 == 0, "parameter slots must stay 16-byte aligned");
+
+struct TShared {
+    unsigned long long full[kTStages];
+    unsigned long long empty[kTStages];
+    int abort;
+};
+
+// The channels of one tile for one consumer warp; returns false when a wait gave up.
+template <int ELL, bool ODD>
+__device__ __forceinline__ bool t_channels(const float* stages, const KRec* rec, const int (&off)[4], uint32_t full0,
+                                           uint32_t empty0, uint32_t& st, int lane, u64 (&acc)[kR]) {
+    const int m = rec->m;
     for (int q = 0; q < m; ++q) {
-        const int slot = q & 1;
-        if (warp == 0 && q + 1 < m)
-            t_issue_stage(Xn + (size_t)kb[10 + q + 1] * a.L, a.plan.zeros, chunks, nch, rows, d, a.L,
-                          smem_u32(stages + (slot ^ 1) * kTStageFloats), bar0 + 8u * (slot ^ 1), lane);
-        if (!mbar_wait(bar0 + 8u * slot, phase[slot])) atomicExch(a.plan.error_flag, 1);
-        phase[slot] ^= 1u;
-        conv_channel<ELL, R, kTPitch>(stages + slot * kTStageFloats, col, wbuf + q * kWeightRow, acc);
-        __syncthreads();  // every warp is done with this slot before it is refilled
+        const uint32_t slot = st % kTStages;
+        if (q > 0 && !mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) return false;
+        conv_channel<ELL, ODD, kTBoxCols>(stages + slot * kTStageFloats, off, rec->w2[q], acc);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8u * slot);
+        ++st;
     }
-    pool_hard<R>(acc, interior, o_lo, o_hi, cnt, mn);
+    return true;
 }
 
 __global__ void __launch_bounds__(kTThreads, 4) fast_t_forward(FwdArgs a) {
-    float* stages = smem;                                   // [2][kRowsMax][kTPitch]
-    float* wbuf = stages + kTStages * kTStageFloats;        // [11 * 12]
-    int* kb = reinterpret_cast<int*>(wbuf + ROCKET_MAX_CHANNELS_PER_KERNEL * kWeightRow);  // [32]
-    __shared__ __align__(8) unsigned long long bars[kTStages];
-    __shared__ TChunk chunks[kTMaxChunks];
-    __shared__ unsigned s_item;
+    __shared__ __align__(8) TShared sh;
+    // dynamic shared memory, aligned to 128 bytes by hand: stages, then parameter slots
+    const uint32_t raw = smem_u32(smem_raw);
+    unsigned char* base = smem_raw + (((raw + 127u) & ~127u) - raw);
+    float* stages = reinterpret_cast<float*>(base);
+    TParams* params = reinterpret_cast<TParams*>(base + (size_t)kTStages * kTStageFloats * 4);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t bar0 = smem_u32(bars);
+    const uint32_t full0 = smem_u32(sh.full), empty0 = smem_u32(sh.empty);
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kTStages; ++i) mbar_init(bar0 + 8u * i, 1);
+        for (int i = 0; i < kTStages; ++i) {
+            mbar_init(full0 + 8u * i, 1);
+            mbar_init(empty0 + 8u * i, kTConsumerWarps);
+        }
+        sh.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    uint32_t phase[kTStages] = {0u, 0u};
+    __syncthreads();
     const unsigned n_items = (unsigned)a.plan.n_titems;
     const unsigned long long total = (unsigned long long)a.N * n_items;
+    volatile int* abort_flag = &sh.abort;
 
-    for (;;) {
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            // a wait that gave up anywhere ends the whole launch early (results are flagged invalid)
-            const bool failed = *reinterpret_cast<volatile int*>(a.plan.error_flag) != 0;
-            s_item = failed ? 0xffffffffu : atomicAdd(a.plan.counters + 1, 1u);
+    if (warp == kTConsumerWarps) {
+        // ---- producer: one lane issues every copy of the block
+        if (lane == 0) {
+            uint32_t st = 0, it = 0;
+            bool ok = true;
+            for (unsigned long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
+                if (*abort_flag) break;
+                const int n = (int)(g / n_items);
+                const TItem* tp = a.plan.titems + (g - (unsigned long long)n * n_items);
+                const int4 w0 = __ldg(reinterpret_cast<const int4*>(tp));
+                const int4 w1 = __ldg(reinterpret_cast<const int4*>(tp) + 1);
+                const int4 w2 = __ldg(reinterpret_cast<const int4*>(tp) + 2);
+                const int tk = w0.x, t0 = w0.y, r0 = w0.z, shape = w0.w;
+                const int d = w1.x, m = w1.z, box_rows = w1.w;
+                const unsigned chw[3] = {(unsigned)w2.x, (unsigned)w2.y, (unsigned)w2.z};
+                TPhase ph[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) ph[k] = t_phase(t0, r0, d, k);
+                const int ngroups = t_shape_colgroups(shape);
+                const uint32_t box_bytes = (uint32_t)box_rows * kTBoxCols * 4u;
+                const uint32_t phase_bytes = (uint32_t)t_phase_floats(box_rows) * 4u;
+                const char* tmap = reinterpret_cast<const char*>(a.plan.tmaps) + (size_t)(2 * tk + shape) * 128;
+                TParams* ps = params + (it % kTParamSlots);
+                for (int q = 0; q < m; ++q) {
+                    const uint32_t slot = st % kTStages;
+                    if (st >= (uint32_t)kTStages && !mbar_wait(empty0 + 8u * slot, ((st / kTStages) - 1u) & 1u)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t bar = full0 + 8u * slot;
+                    uint32_t tx = (uint32_t)ngroups * 4u * box_bytes;
+                    if (q == 0) tx += (uint32_t)sizeof(TParams);
+                    mbar_arrive_expect_tx(bar, tx);
+                    if (q == 0) {
+                        bulk_g2s(smem_u32(&ps->rec), a.plan.krec + w2.w, (uint32_t)sizeof(KRec), bar);
+                        bulk_g2s(smem_u32(&ps->item), tp, (uint32_t)sizeof(TItem), bar);
+                    }
+                    const int ch = (int)((chw[q >> 2] >> (8 * (q & 3))) & 0xffu);
+                    const int z = n * a.C + ch;
+                    const uint32_t dst0 = smem_u32(stages + slot * kTStageFloats);
+                    for (int wc = 0; wc < ngroups; ++wc)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            tma_load_3d(dst0 + (uint32_t)(wc * 4 + k) * phase_bytes, tmap, ph[k].x + kWarpCols * wc,
+                                        ph[k].y, z, bar);
+                    ++st;
+                }
+                ++it;
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicExch(a.plan.error_flag, 1);
+            }
+            // nothing of this block may still be in flight when it exits: every issued stage has
+            // either been consumed or is waited for here (bounded)
+            for (uint32_t back = 1; back <= (uint32_t)kTStages && back <= st; ++back) {
+                const uint32_t s2 = st - back;
+                mbar_wait(full0 + 8u * (s2 % kTStages), (s2 / kTStages) & 1u);
+            }
         }
-        __syncthreads();
-        const unsigned g = s_item;
-        if (g >= total) break;
-        const int n = (int)(g / n_items);
-        const TItem item = a.plan.titems[g - (unsigned)n * n_items];
-        if (warp == 0) kb[lane] = __ldg(reinterpret_cast<const int*>(a.plan.fk + item.fk) + lane);
-        __syncthreads();
-        const int len = kb[0], d = kb[1], m = kb[3], woff = kb[5], korig = kb[6], lo_u = kb[7], hi_u = kb[8];
-        for (int i = threadIdx.x; i < m * kWeightRow; i += kTThreads) wbuf[i] = __ldg(a.plan.negw + woff + i);
-        const int R = item.R;
-        // chunks of the tile (every thread computes them; thread 0 publishes them for the fill)
-        TChunk my_chunks[kTMaxChunks];
-        int ncols;
-        const int nch = t_make_chunks(item, d, my_chunks, ncols);
-        if (threadIdx.x == 0)
-            for (int i = 0; i < nch; ++i) chunks[i] = my_chunks[i];
-        const TColumn tc = t_column(my_chunks, nch, ncols, d, threadIdx.x);
-        const bool lane_ok = tc.ok;
-        const int u0 = tc.u0;
-        const int col[4] = {tc.col[0], tc.col[1], tc.col[2], tc.col[3]};
-        const bool mine = lane_ok && u0 >= lo_u && (u0 + (R - 1) * d) < hi_u;
-        const bool interior = __all_sync(kFull, mine);
-        int o_lo = 0, o_hi = R;
-        if (!interior) valid_rows(u0, d, lo_u, hi_u, R, lane_ok, o_lo, o_hi);
-        __syncthreads();  // kb, wbuf, chunks visible to everyone
-        const float* __restrict__ Xn = a.X + (size_t)n * a.C * a.L;
-        if (warp == 0)
-            t_issue_stage(Xn + (size_t)kb[10] * a.L, a.plan.zeros, chunks, nch, R + len - 1, d, a.L,
-                          smem_u32(stages), bar0, lane);
-        int cnt = 0;
-        float mn = __int_as_float(0x7f800000);
-#define ROCKET_T_CASE(ELL_, R_)                                                                               \
-    t_kernel_tile<ELL_, R_>(a, stages, wbuf, kb, chunks, nch, Xn, col, bar0, phase, interior, o_lo, o_hi, cnt, mn)
-#define ROCKET_T_LEN(R_)                                                          \
-    do {                                                                          \
-        if (len == 7) ROCKET_T_CASE(7, R_);                                       \
-        else if (len == 9) ROCKET_T_CASE(9, R_);                                  \
-        else ROCKET_T_CASE(11, R_);                                               \
-    } while (0)
-        if (R == 32) ROCKET_T_LEN(32);
-        else if (R == 24) ROCKET_T_LEN(24);
-        else if (R == 16) ROCKET_T_LEN(16);
-        else ROCKET_T_LEN(8);
-#undef ROCKET_T_LEN
-#undef ROCKET_T_CASE
-        publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
+    } else {
+        // ---- consumers
+        uint32_t st = 0, it = 0;
+        bool ok = true;
+        for (unsigned long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
+            if (*abort_flag) break;
+            const int n = (int)(g / n_items);
+            const uint32_t slot = st % kTStages;
+            if (!mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) {
+                ok = false;
+                break;
+            }
+            const TParams* ps = params + (it % kTParamSlots);
+            const KRec* rec = &ps->rec;
+            const int t0 = ps->item.t0, r0 = ps->item.r0, shape = ps->item.shape, box_rows = ps->item.box_rows;
+            const int len = rec->len, d = rec->d, korig = rec->k, lo_u = rec->lo_u, hi_u = rec->hi_u;
+            const int wr = shape == 0 ? warp : (warp >> 1), wc = shape == 0 ? 0 : (warp & 1);
+            const int lc = kWarpCols * wc + 2 * lane;
+            const bool ok0 = r0 + lc < d, ok1 = r0 + lc + 1 < d;
+            const int u00 = (t0 + kR * wr) * d + r0 + lc, u01 = u00 + 1;
+            const bool mine = ok0 && ok1 && u00 >= lo_u && (u01 + (kR - 1) * d) < hi_u;
+            const bool interior = __all_sync(kFull, mine);
+            int lo0 = 0, hi0 = kR, lo1 = 0, hi1 = kR;
+            if (!interior) {
+                valid_rows(u00, d, lo_u, hi_u, kR, ok0, lo0, hi0);
+                valid_rows(u01, d, lo_u, hi_u, kR, ok1, lo1, hi1);
+            }
+            int off[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                off[k] = t_box_offset(wc, k, box_rows) + 4 * wr * kTBoxCols + (((t0 + k) * d) & 3) + 2 * lane;
+            u64 acc[kR];
+            const u64 negb = pack2(rec->negb, rec->negb);
+#pragma unroll
+            for (int o = 0; o < kR; ++o) acc[o] = negb;
+            const bool odd = (d & 1) != 0;
+            if (len == 7) ok = odd ? t_channels<7, true>(stages, rec, off, full0, empty0, st, lane, acc)
+                                   : t_channels<7, false>(stages, rec, off, full0, empty0, st, lane, acc);
+            else if (len == 9) ok = odd ? t_channels<9, true>(stages, rec, off, full0, empty0, st, lane, acc)
+                                        : t_channels<9, false>(stages, rec, off, full0, empty0, st, lane, acc);
+            else ok = odd ? t_channels<11, true>(stages, rec, off, full0, empty0, st, lane, acc)
+                          : t_channels<11, false>(stages, rec, off, full0, empty0, st, lane, acc);
+            if (!ok) break;
+            int cnt = 0;
+            float mn = __int_as_float(0x7f800000);
+            pool_hard(acc, interior, lo0, hi0, lo1, hi1, cnt, mn);
+            publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
+            ++it;
+        }
+        if (!ok) {
+            *abort_flag = 1;
+            if (lane == 0) atomicExch(a.plan.error_flag, 1);
+        }
     }
+    __syncthreads();  // every wait above is bounded, so every warp gets here
 }
 
 // ------------------------------------------------------------------------------------------------
-// init / finalise
+// pad copy / init / finalise
 // ------------------------------------------------------------------------------------------------
+__global__ void fast_pad_copy_kernel(const float4* __restrict__ X, float4* __restrict__ xpad, int64_t rows, int L4,
+                                     int64_t pitch4, int front4) {
+    const int64_t total = rows * L4;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t rho = e / L4;
+        const int i = (int)(e - rho * L4);
+        xpad[rho * pitch4 + front4 + i] = __ldg(X + e);
+    }
+}
+
 __global__ void fast_init_kernel(int* __restrict__ feat_i, int64_t pairs, unsigned* counters) {
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e == 0) { counters[0] = 0u; counters[1] = 0u; }
     if (e < pairs) { feat_i[2 * e] = 0; feat_i[2 * e + 1] = INT_MIN; }
 }
 
-__global__ void fast_finalize_kernel(float* __restrict__ feat, const FastKernel* __restrict__ fk, int n_fk, int N,
+__global__ void fast_finalize_kernel(float* __restrict__ feat, const KRec* __restrict__ krec, int n_krec, int N,
                                      int K) {
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= (int64_t)N * n_fk) return;
-    const int n = (int)(e / n_fk), f = (int)(e - (int64_t)n * n_fk);
-    const int k = fk[f].k, nout = fk[f].nout;
+    if (e >= (int64_t)N * n_krec) return;
+    const int n = (int)(e / n_krec), f = (int)(e - (int64_t)n * n_krec);
+    const int k = krec[f].k, nout = krec[f].nout;
     int* fi = reinterpret_cast<int*>(feat) + ((int64_t)n * K + k) * 2;
     const int cnt = fi[0], key = fi[1];
     feat[((int64_t)n * K + k) * 2] = (float)cnt / (float)nout;   // Eq. 2
     feat[((int64_t)n * K + k) * 2 + 1] = key_float(key);
 }
 
+size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+size_t s_smem_bytes(int C) { return (size_t)C * kSPlaneFloats * 4 + (size_t)kSWarps * 2 * sizeof(KRec); }
+size_t t_smem_bytes() { return (size_t)kTStages * kTStageFloats * 4 + (size_t)kTParamSlots * sizeof(TParams) + 128; }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
 }  // namespace
 
-size_t s_smem_bytes(int C) {
-    return (size_t)(C * kSPlaneFloats + kSWarps * ROCKET_MAX_CHANNELS_PER_KERNEL * kWeightRow + kSWarps * 32) * 4;
-}
-size_t t_smem_bytes() {
-    return (size_t)(kTStages * kTStageFloats + ROCKET_MAX_CHANNELS_PER_KERNEL * kWeightRow + 32) * 4;
+cudaError_t upload_plan(FastState& fs) {
+    const PlanHost& h = fs.host;
+    PlanDevice& d = fs.dev;
+    d = PlanDevice();
+    struct Part { const void* src; size_t bytes; size_t off; };
+    Part parts[7] = {
+        {h.krec.data(), h.krec.size() * sizeof(KRec), 0},   {h.sb.data(), h.sb.size() * sizeof(SBucket), 0},
+        {h.sitems.data(), h.sitems.size() * sizeof(SItem), 0}, {h.titems.data(), h.titems.size() * sizeof(TItem), 0},
+        {h.generic_list.data(), h.generic_list.size() * 4, 0}, {nullptr, 256, 0}, {nullptr, 256, 0}};
+    size_t total = 0;
+    for (auto& pt : parts) { pt.off = total; total += align256(pt.bytes); }
+    cudaError_t e = cudaMalloc(&fs.plan_blob, std::max<size_t>(total, 256));
+    if (e != cudaSuccess) { fs.plan_blob = nullptr; return e; }
+    char* base = static_cast<char*>(fs.plan_blob);
+    e = cudaMemset(base, 0, std::max<size_t>(total, 256));
+    for (auto& pt : parts)
+        if (e == cudaSuccess && pt.src && pt.bytes) e = cudaMemcpy(base + pt.off, pt.src, pt.bytes, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) { cudaFree(fs.plan_blob); fs.plan_blob = nullptr; return e; }
+    d.krec = reinterpret_cast<const KRec*>(base + parts[0].off);
+    d.sb = reinterpret_cast<const SBucket*>(base + parts[1].off);
+    d.sitems = reinterpret_cast<const SItem*>(base + parts[2].off);
+    d.titems = reinterpret_cast<const TItem*>(base + parts[3].off);
+    d.generic_list = reinterpret_cast<const int32_t*>(base + parts[4].off);
+    d.counters = reinterpret_cast<unsigned*>(base + parts[5].off);
+    d.error_flag = reinterpret_cast<int*>(base + parts[6].off);
+    d.n_krec = (int)h.krec.size(); d.n_sitems = (int)h.sitems.size(); d.n_titems = (int)h.titems.size();
+    d.n_generic = (int)h.generic_list.size(); d.n_tkernels = (int)h.tkernels.size();
+    d.pad_pitch = h.pad_pitch;
+    return cudaSuccess;
 }
 
-cudaError_t launch_fast_forward(const PlanDevice& pd, const DeviceParams& dp, const float* X, int N, float* feat,
+void release_fast_state(FastState& fs) {
+    if (fs.plan_blob) cudaFree(fs.plan_blob);
+    if (fs.maps_blob) cudaFree(fs.maps_blob);
+    if (fs.xpad) cudaFree(fs.xpad);
+    fs.plan_blob = fs.maps_blob = nullptr;
+    fs.xpad = nullptr;
+    fs.pad_examples = 0;
+}
+
+cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L) {
+    if (fs.host.tkernels.empty() || N <= fs.pad_examples) return cudaSuccess;
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return cudaErrorNotSupported;
+    const int64_t pitch = fs.host.pad_pitch, rows = (int64_t)N * C;
+    const size_t bytes = (size_t)(rows + 1) * (size_t)pitch * 4;
+    if (fs.xpad) cudaFree(fs.xpad);  // waits for work that still reads it
+    fs.xpad = nullptr;
+    fs.pad_examples = 0;
+    cudaError_t e = cudaMalloc(&fs.xpad, bytes);
+    if (e != cudaSuccess) { fs.xpad = nullptr; return e; }
+    e = cudaMemset(fs.xpad, 0, bytes);  // the margins stay zero from here on: the pad copy writes samples only
+    if (e != cudaSuccess) return e;
+    const size_t n_maps = 2 * fs.host.tkernels.size();
+    std::vector<CUtensorMap> maps(n_maps);
+    for (size_t i = 0; i < fs.host.tkernels.size(); ++i) {
+        const KRec& f = fs.host.krec[fs.host.tkernels[i]];
+        for (int shape = 0; shape < 2; ++shape) {
+            const cuuint64_t run = 4ull * (cuuint64_t)f.d;
+            const cuuint64_t dims[3] = {run + kTXExtra, ((cuuint64_t)kTPadFront + (cuuint64_t)L + run - 1) / run,
+                                        (cuuint64_t)rows};
+            const cuuint64_t strides[2] = {run * 4ull, (cuuint64_t)pitch * 4ull};
+            const cuuint32_t box[3] = {(cuuint32_t)kTBoxCols, (cuuint32_t)t_box_rows(shape, f.len), 1u};
+            const cuuint32_t elem[3] = {1u, 1u, 1u};
+            const CUresult r = encode(&maps[2 * i + shape], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, fs.xpad, dims, strides, box,
+                                      elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                      CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+        }
+    }
+    static_assert(sizeof(CUtensorMap) == 128, "tensor maps are addressed in 128-byte steps");
+    if (!fs.maps_blob) {
+        e = cudaMalloc(&fs.maps_blob, n_maps * sizeof(CUtensorMap));
+        if (e != cudaSuccess) { fs.maps_blob = nullptr; return e; }
+    }
+    e = cudaMemcpy(fs.maps_blob, maps.data(), n_maps * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) return e;
+    fs.pad_examples = N;
+    fs.dev.tmaps = fs.maps_blob;
+    fs.dev.xpad = fs.xpad;
+    return cudaSuccess;
+}
+
+cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const float* X, int N, float* feat,
                                 cudaStream_t stream) {
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    static bool attr_done = false;
+    static bool attr_done_for[64] = {};
+    bool& attr_done = attr_done_for[dev & 63];
     const size_t s_bytes = s_smem_bytes(dp.C), t_bytes = t_smem_bytes();
     if (!attr_done) {
         e = cudaFuncSetAttribute(fast_s_forward, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s_smem_bytes(kSMaxChannels));
@@ -391,15 +616,27 @@ cudaError_t launch_fast_forward(const PlanDevice& pd, const DeviceParams& dp, co
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
+    const PlanDevice& pd = fs.dev;
+    if (pd.n_titems > 0) {
+        e = ensure_pad_capacity(fs, N, dp.C, dp.L);
+        if (e != cudaSuccess) return e;
+    }
     FwdArgs a;
-    a.plan = pd; a.X = X; a.feat_i = reinterpret_cast<int*>(feat);
+    a.plan = fs.dev; a.X = X; a.feat_i = reinterpret_cast<int*>(feat);
     a.N = N; a.C = dp.C; a.L = dp.L; a.K = dp.K;
     const int64_t pairs = (int64_t)N * dp.K;
     fast_init_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, stream>>>(a.feat_i, pairs, pd.counters);
     count_launch();
+    if (pd.n_titems > 0) {
+        const int64_t rows = (int64_t)N * dp.C;
+        fast_pad_copy_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(X),
+                                                          reinterpret_cast<float4*>(fs.xpad), rows, dp.L / 4,
+                                                          fs.host.pad_pitch / 4, kTPadFront / 4);
+        count_launch();
+    }
     if (pd.n_sitems > 0) {
         const unsigned long long total = (unsigned long long)N * pd.n_sitems;
-        const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms * 2);
+        const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms);
         fast_s_forward<<<grid, kSThreads, s_bytes, stream>>>(a);
         count_launch();
     }
@@ -409,9 +646,9 @@ cudaError_t launch_fast_forward(const PlanDevice& pd, const DeviceParams& dp, co
         fast_t_forward<<<grid, kTThreads, t_bytes, stream>>>(a);
         count_launch();
     }
-    const int64_t fin = (int64_t)N * pd.n_fk;
+    const int64_t fin = (int64_t)N * pd.n_krec;
     if (fin > 0) {
-        fast_finalize_kernel<<<(unsigned)((fin + 255) / 256), 256, 0, stream>>>(feat, pd.fk, pd.n_fk, N, dp.K);
+        fast_finalize_kernel<<<(unsigned)((fin + 255) / 256), 256, 0, stream>>>(feat, pd.krec, pd.n_krec, N, dp.K);
         count_launch();
     }
     return cudaGetLastError();

@@ -55,7 +55,7 @@ cudaError_t launch_generic_backward(const DeviceParams& dp, int64_t n_weights, c
 
 }  // namespace rocket
 
-namespace rocket { namespace fast { struct PlanHost; struct PlanDevice; } }
+namespace rocket { namespace fast { struct FastState; } }
 
 // Grow-only device buffer owned by a handle.
 struct DeviceBuffer {
@@ -81,9 +81,7 @@ struct rocket_params {
     mutable void* dev_blob = nullptr;  // one allocation holding every parameter array
     mutable rocket::DeviceParams dp{};
     mutable DeviceBuffer scratch; // backward partial sums
-    rocket::fast::PlanHost* plan_host = nullptr;              // fast-path launch plan (host copy)
-    mutable rocket::fast::PlanDevice* plan_dev = nullptr;     // its device pointers, filled at binding
-    mutable void* plan_blob = nullptr;                        // one allocation holding the device plan
+    rocket::fast::FastState* fast = nullptr;   // fast-path launch plan and its device-side state
     DeviceBuffer stage_x, stage_feat, stage_arg, stage_g, stage_dw;  // host-call staging
     cudaStream_t host_stream = nullptr;
 };

@@ -1,5 +1,5 @@
 // Host-side launch plan of the fast path: buckets kernels by dilation, lays out band rasters,
-// cuts them into tiles and orders the tiles by cost (largest first) for the persistent kernels.
+// cuts them into tiles and orders the tiles by cost (largest first).
 #include <algorithm>
 #include <map>
 
@@ -15,11 +15,11 @@ inline int64_t floor_div(int64_t a, int64_t b) { return (a >= 0) ? a / b : -((-a
 
 void build_plan(const HostParams& hp, int split, PlanHost& out) {
     out = PlanHost();
-    if (split < 64) split = 64;  // T tiles need d >= 64 so that a 128-column tile spans at most 3 bands
+    if (split < kTMinDilation) split = kTMinDilation;
     out.split = split;
     const int K = hp.K;
-    // The fast kernels want 16-byte aligned channel rows (bulk copies) and at most
-    // kSMaxChannels channels in an S tile.
+    // The fast kernels want 16-byte aligned channel rows and at most kSMaxChannels channels in
+    // an S tile.
     const bool shape_ok = (hp.L % 4 == 0) && hp.C <= kSMaxChannels && hp.L >= 16;
     std::vector<int> s_kernels, t_kernels;
     for (int k = 0; k < K; ++k) {
@@ -33,21 +33,18 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
     if (!out.enabled) return;
 
     auto add_kernel = [&](int k) {
-        FastKernel f{};
+        KRec f{};
         f.len = hp.length[k]; f.d = hp.dilation[k]; f.p = hp.padding[k]; f.m = hp.num_channels[k];
         f.nout = (int32_t)((int64_t)hp.L + 2 * (int64_t)f.p - (int64_t)(f.len - 1) * f.d);
-        f.woff = (int32_t)out.negw.size();
         f.k = k; f.lo_u = -f.p; f.hi_u = f.nout - f.p;
         f.negb = 0.0f - hp.bias[k];
         const int32_t* S = hp.channel_idx.data() + hp.channel_offset[k];
         const float* W = hp.weights.data() + hp.weight_offset[k];
-        // weights of fast kernel i live at negw[i * kWeightsPerKernel], rows padded to kWeightRow
-        out.negw.resize(out.negw.size() + kWeightsPerKernel, 0.0f);
         for (int q = 0; q < f.m; ++q) {
             f.ch[q] = S[q];
-            for (int j = 0; j < f.len; ++j) out.negw[f.woff + q * kWeightRow + j] = 0.0f - W[q * f.len + j];
+            for (int j = 0; j < f.len; ++j) f.w2[q][2 * j] = f.w2[q][2 * j + 1] = 0.0f - W[q * f.len + j];
         }
-        out.fk.push_back(f);
+        out.krec.push_back(f);
     };
 
     // ---- S regime: one bucket per dilation, kernels inside ordered by cost (largest first)
@@ -62,27 +59,27 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
             return hp.length[a] * hp.num_channels[a] > hp.length[b] * hp.num_channels[b];
         });
         SBucket b{};
-        b.d = d; b.kbeg = (int32_t)out.fk.size();
+        b.d = d; b.kbeg = (int32_t)out.krec.size();
         int64_t tmin = INT64_MAX, tmax = INT64_MIN;
         int maxlen = 0;
         double work = 0.0;
         for (int k : ks) {
             add_kernel(k);
-            const FastKernel& f = out.fk.back();
+            const KRec& f = out.krec.back();
             tmin = std::min(tmin, floor_div(f.lo_u, d));
             tmax = std::max(tmax, floor_div((int64_t)f.hi_u - 1, d));
             maxlen = std::max(maxlen, f.len);
-            work += (double)f.len * f.m;
+            work += (double)f.m * (f.len + 2) + 6.0;
         }
-        b.kend = (int32_t)out.fk.size();
+        b.kend = (int32_t)out.krec.size();
         b.tmin = (int32_t)tmin;
-        b.nbands = (int32_t)((tmax - tmin + 1 + kBandRows - 1) / kBandRows);
+        b.nbands = (int32_t)((tmax - tmin + 1 + kR - 1) / kR);
         b.raster_len = b.nbands * d;
-        b.rows = kBandRows + maxlen - 1;
+        b.rows = kR + maxlen - 1;
         const int bi = (int)out.sb.size();
         out.sb.push_back(b);
-        for (int c0 = 0; c0 < b.raster_len; c0 += kSCols) {
-            s_cost.push_back({work + 0.02 * hp.C * b.rows, (int)out.sitems.size()});
+        for (int c0 = 0; c0 < b.raster_len; c0 += kWarpCols) {
+            s_cost.push_back({work + 0.3 * hp.C * b.rows, (int)out.sitems.size()});
             out.sitems.push_back({bi, c0});
         }
     }
@@ -94,25 +91,37 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         out.sitems.swap(sorted);
     }
 
-    // ---- T regime: per kernel, full bands of 32 rows and one tail band of 8/16/24/32 rows
+    // ---- T regime: per kernel, bands of 64 rows (shape 0) and a last band of 32 (shape 1) or 64
     std::vector<Cost> t_cost;
+    int d_max = 0;
     for (int k : t_kernels) {
-        const int fi = (int)out.fk.size();
+        const int ki = (int)out.krec.size();
         add_kernel(k);
-        const FastKernel f = out.fk.back();
-        const int64_t tmin = floor_div(f.lo_u, f.d), tmax = floor_div((int64_t)f.hi_u - 1, f.d);
+        const KRec f = out.krec.back();
+        const int tk = (int)out.tkernels.size();
+        out.tkernels.push_back(ki);
+        d_max = std::max(d_max, f.d);
+        int64_t tmin = floor_div(f.lo_u, f.d);
+        const int64_t tmax = floor_div((int64_t)f.hi_u - 1, f.d);
+        // odd dilations: an even first row keeps the rows of phases 0 and 2 aligned to pairs
+        if (f.d & 1) tmin = floor_div(tmin, 2) * 2;
         const int64_t rows = tmax - tmin + 1;
-        const int64_t nb = rows / kBandRows, rem = rows % kBandRows;
-        auto add_group = [&](int64_t t0, int R, int64_t raster_len) {
-            for (int64_t c0 = 0; c0 < raster_len; c0 += kTCols) {
+        auto add_band = [&](int64_t t0, int shape) {
+            const int cols = kWarpCols * t_shape_colgroups(shape);
+            for (int r0 = 0; r0 < f.d; r0 += cols) {
                 TItem it{};
-                it.fk = fi; it.t0 = (int32_t)t0; it.R = R; it.c0 = (int32_t)c0; it.raster_len = (int32_t)raster_len;
-                t_cost.push_back({(double)f.len * f.m * (R + 3.0) + 40.0, (int)out.titems.size()});
+                it.tk = tk; it.t0 = (int32_t)t0; it.r0 = r0; it.shape = shape;
+                it.d = f.d; it.len = f.len; it.m = f.m; it.box_rows = t_box_rows(shape, f.len);
+                for (int q = 0; q < f.m; ++q) it.ch[q] = (uint8_t)f.ch[q];
+                it.krec = ki;
+                t_cost.push_back({(double)f.m * (f.len + 2) + 6.0, (int)out.titems.size()});
                 out.titems.push_back(it);
             }
         };
-        if (nb > 0) add_group(tmin, kBandRows, nb * f.d);
-        if (rem > 0) add_group(tmin + nb * kBandRows, (int)((rem + 7) / 8 * 8), f.d);
+        const int64_t full = rows / 64, rem = rows % 64;
+        for (int64_t b = 0; b < full; ++b) add_band(tmin + 64 * b, 0);
+        if (rem > 32) add_band(tmin + 64 * full, 0);
+        else if (rem > 0) add_band(tmin + 64 * full, 1);
     }
     {
         std::stable_sort(t_cost.begin(), t_cost.end(), [](const Cost& a, const Cost& b) { return a.c > b.c; });
@@ -121,6 +130,10 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         for (auto& c : t_cost) sorted.push_back(out.titems[c.idx]);
         out.titems.swap(sorted);
     }
+    // every channel row of the zero-margined copy: front zeros, L samples, zeros for the run a box may
+    // read past the last sample; rounded to 128 bytes
+    const int64_t pitch = (int64_t)kTPadFront + hp.L + 4ll * d_max + kTXExtra + kTBoxCols;
+    out.pad_pitch = (pitch + 31) / 32 * 32;
 }
 
 }  // namespace fast

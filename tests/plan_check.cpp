@@ -1,8 +1,10 @@
 // Host-side checker of the fast path's launch plan and index arithmetic (no GPU needed).
 // For a set of (seed, K, C, L) it builds the plan and replays, with the same integer functions
-// the kernels use, which outputs every thread of every tile owns and which bulk copies every
-// tile issues.  It fails (exit 1) unless every output of every fast kernel is owned exactly once
-// and every copy stays inside its source row and its shared-memory slot with 16-byte alignment.
+// the kernels use, which outputs every thread of every tile owns and which boxes every T tile
+// loads.  It fails (exit 1) unless every output of every fast kernel is owned exactly once, every
+// box obeys the TMA rules (16-byte aligned x, 128-byte aligned destination inside the stage,
+// reads inside the channel row of the zero-margined copy) and every shared-memory word a
+// consumer thread reads holds the sample it expects (or a zero outside the series).
 #include <cstdio>
 #include <cstdlib>
 #include <vector>
@@ -37,25 +39,33 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
     }
     PlanHost plan;
     build_plan(hp, split, plan);
-    std::vector<std::vector<uint8_t>> cover(plan.fk.size());
-    for (size_t f = 0; f < plan.fk.size(); ++f) cover[f].assign(plan.fk[f].nout, 0);
+    std::vector<std::vector<uint8_t>> cover(plan.krec.size());
+    for (size_t f = 0; f < plan.krec.size(); ++f) cover[f].assign(plan.krec[f].nout, 0);
     std::vector<char> is_generic(hp.K, 0);
     for (int k : plan.generic_list) is_generic[k] = 1;
-    REQUIRE(plan.fk.size() + plan.generic_list.size() == (size_t)hp.K, "kernel partition");
-    for (auto& f : plan.fk) REQUIRE(!is_generic[f.k], "kernel %d in both lists", f.k);
+    REQUIRE(plan.krec.size() + plan.generic_list.size() == (size_t)hp.K, "kernel partition");
+    for (auto& f : plan.krec) {
+        REQUIRE(!is_generic[f.k], "kernel %d in both lists", f.k);
+        const float* W = hp.weights.data() + hp.weight_offset[f.k];
+        for (int q = 0; q < f.m; ++q)
+            for (int j = 0; j < kPairRow / 2; ++j) {
+                const float want = j < f.len ? 0.0f - W[q * f.len + j] : 0.0f;
+                REQUIRE(f.w2[q][2 * j] == want && f.w2[q][2 * j + 1] == want, "weight pair");
+            }
+    }
 
     for (const SItem& it : plan.sitems) {
         const SBucket& b = plan.sb[it.bucket];
-        REQUIRE(b.rows <= kRowsMax && b.d < plan.split, "S bucket shape");
-        for (int lane = 0; lane < kSCols; ++lane) {
-            const int cg = it.c0 + lane;
-            const bool lane_ok = cg < b.raster_len;
+        REQUIRE(b.rows <= kRowsMax && b.d < plan.split && it.c0 % kWarpCols == 0, "S bucket shape");
+        for (int col = 0; col < kWarpCols; ++col) {
+            const int cg = it.c0 + col;
+            const bool col_ok = cg < b.raster_len;
             const int u0 = s_column_u0(b, cg);
             for (int kk = b.kbeg; kk < b.kend; ++kk) {
-                const FastKernel& f = plan.fk[kk];
-                REQUIRE(f.d == b.d && kBandRows + f.len - 1 <= b.rows, "S kernel in wrong bucket");
+                const KRec& f = plan.krec[kk];
+                REQUIRE(f.d == b.d && kR + f.len - 1 <= b.rows, "S kernel in wrong bucket");
                 int o_lo, o_hi;
-                valid_rows(u0, b.d, f.lo_u, f.hi_u, kBandRows, lane_ok, o_lo, o_hi);
+                valid_rows(u0, b.d, f.lo_u, f.hi_u, kR, col_ok, o_lo, o_hi);
                 for (int o = o_lo; o < o_hi; ++o) {
                     const int64_t i = (int64_t)u0 + (int64_t)o * b.d + f.p;
                     REQUIRE(i >= 0 && i < f.nout, "S output out of range");
@@ -64,60 +74,81 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
             }
         }
     }
+
+    const int64_t pitch = plan.pad_pitch;
+    REQUIRE(plan.titems.empty() || (pitch % 32 == 0 && pitch >= kTPadFront + L), "pad pitch");
     for (const TItem& it : plan.titems) {
-        const FastKernel& f = plan.fk[it.fk];
-        REQUIRE(f.d >= 64 && (it.R == 8 || it.R == 16 || it.R == 24 || it.R == 32), "T item shape");
-        const int rows = it.R + f.len - 1;
-        REQUIRE(rows <= kRowsMax, "T rows");
-        TChunk chunks[kTMaxChunks];
-        int ncols;
-        const int nch = t_make_chunks(it, f.d, chunks, ncols);
-        REQUIRE(nch >= 1 && nch <= kTMaxChunks && ncols >= 1, "T chunks");
-        for (int c = 0; c < nch; ++c) {
-            const int slot_end = (c + 1 < nch) ? chunks[c + 1].off : kTPitch;
-            REQUIRE(chunks[c].off % 4 == 0 && chunks[c].off + ((chunks[c].w + 3) & ~3) + 4 <= slot_end, "chunk slot");
-        }
-        for (int task = 0; task < nch * rows; ++task) {
-            const TCopy cp = t_copy_of(task, chunks, rows, f.d, L);
-            REQUIRE(cp.tot_bytes % 16 == 0 && cp.in_bytes % 16 == 0 && cp.in_bytes > 0 && cp.in_bytes <= cp.tot_bytes, "copy size");
-            REQUIRE(cp.dst_bytes % 16 == 0 && cp.dst_bytes + cp.tot_bytes <= (uint32_t)kTStageFloats * 4, "copy dst");
-            REQUIRE(cp.tot_bytes - cp.in_bytes <= (uint32_t)kZeroFloats * 4 && cp.tot_bytes <= (uint32_t)kZeroFloats * 4, "zero page");
-            if (cp.src_elem >= 0)
-                REQUIRE(cp.src_elem % 4 == 0 && (int64_t)cp.src_elem + cp.in_bytes / 4 <= L, "copy src %d + %u > %d", cp.src_elem, cp.in_bytes / 4, L);
-        }
-        for (int lc = 0; lc < kTCols; ++lc) {
-            const TColumn tc = t_column(chunks, nch, ncols, f.d, lc);
-            int o_lo, o_hi;
-            valid_rows(tc.u0, f.d, f.lo_u, f.hi_u, it.R, tc.ok, o_lo, o_hi);
-            for (int o = o_lo; o < o_hi; ++o) {
-                const int64_t i = (int64_t)tc.u0 + (int64_t)o * f.d + f.p;
-                REQUIRE(i >= 0 && i < f.nout, "T output out of range");
-                cover[it.fk][i]++;
+        const KRec& f = plan.krec[it.krec];
+        REQUIRE(plan.tkernels[it.tk] == it.krec, "T kernel index");
+        REQUIRE(f.d >= kTMinDilation && f.d == it.d && f.len == it.len && f.m == it.m, "T item fields");
+        REQUIRE(it.shape == 0 || it.shape == 1, "T shape");
+        REQUIRE(it.r0 % kWarpCols == 0 && it.r0 < f.d, "T column origin");
+        REQUIRE(!(f.d & 1) || (it.t0 % 2 == 0), "odd dilation needs an even first row");
+        for (int q = 0; q < f.m; ++q) REQUIRE(it.ch[q] == f.ch[q], "T channel list");
+        const int rows_out = t_shape_rows(it.shape), groups = t_shape_colgroups(it.shape);
+        const int rows = rows_out + f.len - 1;
+        REQUIRE(it.box_rows == t_box_rows(it.shape, f.len) && 4 * it.box_rows >= rows, "T box rows");
+        const long long run = 4ll * f.d, ny = (kTPadFront + (long long)L + run - 1) / run;
+        // the boxes the producer issues
+        TPhase ph[4];
+        for (int k = 0; k < 4; ++k) {
+            ph[k] = t_phase(it.t0, it.r0, f.d, k);
+            REQUIRE(ph[k].x % 4 == 0 && ph[k].x >= 0 && ph[k].x < run, "box x");
+            for (int wc = 0; wc < groups; ++wc) {
+                const int x = ph[k].x + kWarpCols * wc;
+                REQUIRE(x + kTBoxCols <= run + kTXExtra, "box leaves the tensor row");
+                const int dst = t_box_offset(wc, k, it.box_rows);
+                REQUIRE(dst % 32 == 0 && dst + it.box_rows * kTBoxCols <= kTStageFloats, "box destination");
+                for (int j = 0; j < it.box_rows; ++j) {
+                    const long long y = ph[k].y + j;
+                    if (y < 0 || y >= ny) continue;  // zero-filled by the copy engine
+                    const long long first = y * run + x, last = first + kTBoxCols - 1;
+                    REQUIRE(first >= 0 && last < pitch, "box row reads outside its channel row: %lld..%lld of %lld", first,
+                            last, (long long)pitch);
+                }
             }
-            // every row the thread reads lies inside a copied region and holds the element it expects
-            int sel = 0, start = 0, within = lc;
-            for (int c = 0; c < nch; ++c) { if (lc >= start && lc < start + chunks[c].w) { sel = c; within = lc - start; } start += chunks[c].w; }
-            if (!tc.ok) { sel = 0; within = 0; }
-            for (int s = 0; s < rows; ++s) {
-                const int pos = tc.col[s & 3] + s * kTPitch;
-                REQUIRE(pos >= 0 && pos < kTStageFloats, "column read outside the stage");
-                const TCopy cp = t_copy_of(sel * rows + s, chunks, rows, f.d, L);
-                const int rel = pos * 4 - (int)cp.dst_bytes;
-                REQUIRE(rel >= 0 && rel + 4 <= (int)cp.tot_bytes, "column read outside the copied row");
-                const int64_t want = (int64_t)(chunks[sel].tb + s) * f.d + chunks[sel].ra + within;  // x index
-                if (cp.src_elem >= 0 && rel < (int)cp.in_bytes) REQUIRE(cp.src_elem + rel / 4 == want, "wrong element");
-                else REQUIRE(want < 0 || want >= L || cp.src_elem < 0, "zero page where data is expected");
-                if (cp.src_elem < 0) REQUIRE(want < 0 || want >= L || (chunks[sel].tb + s) < 0 ||
-                                             (int64_t)(chunks[sel].tb + s) * f.d + chunks[sel].ra >= L, "zero row misplaced");
+        }
+        // what every consumer thread owns and reads
+        for (int lc = 0; lc < kWarpCols * groups; ++lc) {
+            const bool col_ok = it.r0 + lc < f.d;
+            for (int wr = 0; wr < rows_out / kR; ++wr) {
+                const int u0 = (it.t0 + kR * wr) * f.d + it.r0 + lc;
+                int o_lo, o_hi;
+                valid_rows(u0, f.d, f.lo_u, f.hi_u, kR, col_ok, o_lo, o_hi);
+                for (int o = o_lo; o < o_hi; ++o) {
+                    const int64_t i = (int64_t)u0 + (int64_t)o * f.d + f.p;
+                    REQUIRE(i >= 0 && i < f.nout, "T output out of range");
+                    cover[it.krec][i]++;
+                }
+                if (o_lo >= o_hi) continue;
+                for (int s2 = 0; s2 < kR + f.len - 1; ++s2) {
+                    const int s = kR * wr + s2, k = s & 3;
+                    const int shift = ((it.t0 + k) * f.d) & 3;
+                    REQUIRE(shift == ph[k].shift, "alignment shift");
+                    const int pos = t_elem_offset(s, lc, it.box_rows, shift);
+                    REQUIRE(pos >= 0 && pos < kTStageFloats, "read outside the stage");
+                    if ((lc & 1) == 0) REQUIRE(((f.d & 1) && (s2 & 1)) || pos % 2 == 0, "pair not 8-byte aligned");
+                    // which sample the copy engine put there
+                    const int wc = lc >> 6;
+                    const int rel = pos - t_box_offset(wc, k, it.box_rows);
+                    const int j = rel / kTBoxCols, i = rel % kTBoxCols;
+                    REQUIRE(j < it.box_rows, "read below the box");
+                    const long long y = ph[k].y + j;
+                    const long long flat = y * run + ph[k].x + kWarpCols * wc + i;
+                    const long long want = (long long)kTPadFront + (long long)(it.t0 + s) * f.d + it.r0 + lc;
+                    REQUIRE(flat == want, "wrong sample: got flat %lld, want %lld", flat, want);
+                    const bool in_series = want >= kTPadFront && want < kTPadFront + L;
+                    if (y < 0 || y >= ny) REQUIRE(!in_series, "zero fill where a sample is expected");
+                }
             }
         }
     }
-    for (size_t fidx = 0; fidx < plan.fk.size(); ++fidx)
-        for (int i = 0; i < plan.fk[fidx].nout; ++i)
-            REQUIRE(cover[fidx][i] == 1, "kernel %d (len %d d %d p %d) output %d owned %d times", plan.fk[fidx].k,
-                    plan.fk[fidx].len, plan.fk[fidx].d, plan.fk[fidx].p, i, (int)cover[fidx][i]);
+    for (size_t fidx = 0; fidx < plan.krec.size(); ++fidx)
+        for (int i = 0; i < plan.krec[fidx].nout; ++i)
+            REQUIRE(cover[fidx][i] == 1, "kernel %d (len %d d %d p %d) output %d owned %d times", plan.krec[fidx].k,
+                    plan.krec[fidx].len, plan.krec[fidx].d, plan.krec[fidx].p, i, (int)cover[fidx][i]);
     std::printf("ok seed=%llu K=%d C=%d L=%d split=%d: %zu fast kernels, %zu generic, %zu S items, %zu T items\n",
-                (unsigned long long)seed, hp.K, hp.C, hp.L, plan.split, plan.fk.size(), plan.generic_list.size(),
+                (unsigned long long)seed, hp.K, hp.C, hp.L, plan.split, plan.krec.size(), plan.generic_list.size(),
                 plan.sitems.size(), plan.titems.size());
     return 0;
 }
@@ -141,6 +172,7 @@ int main() {
     };
     add(7, 166, 0); add(7, 166, 498); add(11, 99, 495); add(9, 7, 40); add(7, 64, 5); add(9, 65, 300); add(11, 100, 1);
     add(7, 1, 0); add(7, 1, 3); add(9, 63, 17); add(7, 127, 381); add(7, 128, 0); add(9, 124, 0); add(3, 5, 0); add(5, 70, 3);
+    add(7, 129, 5); add(9, 77, 308); add(11, 91, 2);
     rc |= check(0, hp.K, hp.C, hp.L, 64, &hp);
     return rc;
 }

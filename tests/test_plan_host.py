@@ -1,6 +1,7 @@
 """Runs the host-side plan checker (tests/plan_check.cpp): every output of every fast-path kernel
-is owned by exactly one thread of one tile, and every bulk copy of the fill stays inside its
-source row and its shared-memory slot with 16-byte alignment."""
+is owned by exactly one thread of one tile, every TMA box of the fill obeys the alignment rules and
+stays inside its channel row and its shared-memory stage, and every word a consumer reads holds the
+sample it expects."""
 import os
 import subprocess
 
