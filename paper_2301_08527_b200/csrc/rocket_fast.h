@@ -16,8 +16,8 @@
 //     raster positions, so lanes stay busy even when d < 64.  A block stages one tile of ALL
 //     channels in shared memory, then its warps pull kernels of the bucket from a shared
 //     counter, so one staged tile serves dozens to hundreds of kernels.
-//   T (d >= split): few kernels share a dilation, so a block of four consumer warps takes one
-//     kernel and one tile (64 rows x 64 columns or 32 rows x 128 columns) and streams the
+//   T (d >= split): few kernels share a dilation, so a block of eight consumer warps takes one
+//     kernel and one tile of up to eight warp tiles (128 x 64, 64 x 128 or 32 x 256) and streams the
 //     kernel's channels through a ring of shared-memory stages.  A producer warp fills the
 //     ring with tiled TMA loads from a zero-margined copy of the batch, viewed as a 3-D tensor
 //     (x within a run of 4d floats, y = which run, z = channel row): rows s, s+4, s+8, .. of
@@ -71,33 +71,39 @@ struct SBucket {
 struct SItem { int32_t bucket, c0; };
 
 // ---- T regime --------------------------------------------------------------------------------
-constexpr int kTConsumerWarps = 4;
+constexpr int kTConsumerWarps = 8;
 constexpr int kTThreads = 32 * (kTConsumerWarps + 1);              // + one producer warp
-constexpr int kTBoxCols = kWarpCols + 4;                           // 4 floats of 16-byte alignment slack
 constexpr int kTStages = 2;
 constexpr int kTParamSlots = kTStages + 2;
-// Two tile shapes: shape 0 = 4 row groups x 1 column group (64 x 64 outputs),
-//                  shape 1 = 2 row groups x 2 column groups (32 x 128 outputs).
-ROCKET_CX int t_shape_rows(int shape) { return shape == 0 ? 64 : 32; }
-ROCKET_CX int t_shape_colgroups(int shape) { return shape == 0 ? 1 : 2; }
+// A T tile is rg row groups x cg column groups of warp tiles, rg * cg <= 8, cg in {1, 2, 4}.
+// One box per phase brings one (cg = 1: 64 + 4 floats wide) or two (cg >= 2: 128 + 4 wide)
+// column groups; cg = 4 takes two boxes per phase.
+ROCKET_CX int t_box_cols(int cg) { return cg == 1 ? kWarpCols + 4 : 2 * kWarpCols + 4; }
+ROCKET_CX int t_boxes_per_phase(int cg) { return cg <= 2 ? 1 : 2; }
 // Box rows of one phase (rows s, s+4, ..), and the phase pitch in floats (a multiple of 32
 // floats keeps every box destination 128-byte aligned).
-ROCKET_CX int t_box_rows(int shape, int len) { return (t_shape_rows(shape) + len - 1 + 3) / 4; }
-ROCKET_CX int t_phase_floats(int box_rows) { return (box_rows * kTBoxCols + 31) / 32 * 32; }
-constexpr int kTStageFloats0 = 4 * t_phase_floats(t_box_rows(0, ROCKET_MAX_LENGTH));
-constexpr int kTStageFloats1 = 8 * t_phase_floats(t_box_rows(1, ROCKET_MAX_LENGTH));
-constexpr int kTStageFloats = kTStageFloats0 > kTStageFloats1 ? kTStageFloats0 : kTStageFloats1;
+ROCKET_CX int t_box_rows(int rg, int len) { return (kR * rg + len - 1 + 3) / 4; }
+ROCKET_CX int t_phase_floats(int cg, int box_rows) { return (box_rows * t_box_cols(cg) + 31) / 32 * 32; }
+ROCKET_CX int t_stage_floats(int rg, int cg, int len) {
+    return 4 * t_boxes_per_phase(cg) * t_phase_floats(cg, t_box_rows(rg, len));
+}
+ROCKET_CX int imax_cx(int a, int b) { return a > b ? a : b; }
+constexpr int kTStageFloats = imax_cx(imax_cx(t_stage_floats(8, 1, ROCKET_MAX_LENGTH), t_stage_floats(4, 2, ROCKET_MAX_LENGTH)),
+                                      t_stage_floats(2, 4, ROCKET_MAX_LENGTH));
 constexpr int kTPadFront = 128;                                    // zero floats before every channel row
-constexpr int kTXExtra = 128;                                      // floats a box may run past a 4d run
+constexpr int kTXExtra = 256;                                      // floats a box may run past a 4d run
 
 // One T tile with everything the producer warp needs (16 words).
 struct alignas(16) TItem {
-    int32_t tk, t0, r0, shape;            // tk: index into the T kernel list; tile origin (t0, r0)
+    int32_t map, t0, r0, rg;              // map: index of the tile's tensor map; tile origin (t0, r0)
     int32_t d, len, m, box_rows;
     uint8_t ch[12];
-    int32_t krec, pad_[4];                // krec: index into the kernel records
+    int32_t krec;                         // index into the kernel records
+    int32_t cg, pad_[3];
 };
 static_assert(sizeof(TItem) == 64, "TItem must be 16 words");
+// One tensor map: boxes of box_cols x box_rows floats over runs of 4 * d floats.
+struct TMapSpec { int32_t d, box_cols, box_rows; };
 
 struct PlanHost {
     bool enabled = false;
@@ -106,7 +112,7 @@ struct PlanHost {
     std::vector<SBucket> sb;
     std::vector<SItem> sitems;
     std::vector<TItem> titems;
-    std::vector<int32_t> tkernels;        // krec index of every T kernel (tensor maps 2*i, 2*i+1 belong to it)
+    std::vector<TMapSpec> tmaps;          // tensor maps the T tiles refer to
     std::vector<int32_t> generic_list;    // kernels the fast path does not take
     int64_t pad_pitch = 0;                // floats per channel row of the zero-margined copy
 };
@@ -119,10 +125,10 @@ struct PlanDevice {
     const int32_t* generic_list = nullptr;
     unsigned* counters = nullptr;         // [0] S work counter
     int* error_flag = nullptr;            // set when a bounded wait gave up
-    const void* tmaps = nullptr;          // CUtensorMap[2 * n_tkernels], 128 bytes each
+    const void* tmaps = nullptr;          // CUtensorMap[n_tmaps], 128 bytes each
     float* xpad = nullptr;                // zero-margined copy of the batch
     int64_t pad_pitch = 0;
-    int n_krec = 0, n_sitems = 0, n_titems = 0, n_generic = 0, n_tkernels = 0;
+    int n_krec = 0, n_sitems = 0, n_titems = 0, n_generic = 0, n_tmaps = 0;
 };
 
 // Builds the launch plan for the kernels in hp (host side, once per handle).

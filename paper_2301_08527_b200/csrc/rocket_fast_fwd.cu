@@ -307,15 +307,16 @@ struct TShared {
     int abort;
 };
 
-// The channels of one tile for one consumer warp; returns false when a wait gave up.
-template <int ELL, bool ODD>
+// The channels of one tile for one consumer warp; returns false when a wait gave up.  A warp
+// without a valid output (active == false) only keeps the ring moving.
+template <int ELL, bool ODD, int STEP>
 __device__ __forceinline__ bool t_channels(const float* stages, const KRec* rec, const int (&off)[4], uint32_t full0,
-                                           uint32_t empty0, uint32_t& st, int lane, u64 (&acc)[kR]) {
+                                           uint32_t empty0, uint32_t& st, int lane, bool active, u64 (&acc)[kR]) {
     const int m = rec->m;
     for (int q = 0; q < m; ++q) {
         const uint32_t slot = st % kTStages;
         if (q > 0 && !mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) return false;
-        conv_channel<ELL, ODD, kTBoxCols>(stages + slot * kTStageFloats, off, rec->w2[q], acc);
+        if (active) conv_channel<ELL, ODD, STEP>(stages + slot * kTStageFloats, off, rec->w2[q], acc);
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * slot);
         ++st;
@@ -323,7 +324,19 @@ __device__ __forceinline__ bool t_channels(const float* stages, const KRec* rec,
     return true;
 }
 
-__global__ void __launch_bounds__(kTThreads, 4) fast_t_forward(FwdArgs a) {
+template <int STEP>
+__device__ __forceinline__ bool t_dispatch(int len, bool odd, const float* stages, const KRec* rec, const int (&off)[4],
+                                           uint32_t full0, uint32_t empty0, uint32_t& st, int lane, bool active,
+                                           u64 (&acc)[kR]) {
+    if (len == 7) return odd ? t_channels<7, true, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc)
+                             : t_channels<7, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
+    if (len == 9) return odd ? t_channels<9, true, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc)
+                             : t_channels<9, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
+    return odd ? t_channels<11, true, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc)
+               : t_channels<11, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
+}
+
+__global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
     __shared__ __align__(8) TShared sh;
     // dynamic shared memory, aligned to 128 bytes by hand: stages, then parameter slots
     const uint32_t raw = smem_u32(smem_raw);
@@ -357,16 +370,17 @@ __global__ void __launch_bounds__(kTThreads, 4) fast_t_forward(FwdArgs a) {
                 const int4 w0 = __ldg(reinterpret_cast<const int4*>(tp));
                 const int4 w1 = __ldg(reinterpret_cast<const int4*>(tp) + 1);
                 const int4 w2 = __ldg(reinterpret_cast<const int4*>(tp) + 2);
-                const int tk = w0.x, t0 = w0.y, r0 = w0.z, shape = w0.w;
+                const int cg = __ldg(reinterpret_cast<const int*>(tp) + 12);
+                const int map = w0.x, t0 = w0.y, r0 = w0.z;
                 const int d = w1.x, m = w1.z, box_rows = w1.w;
                 const unsigned chw[3] = {(unsigned)w2.x, (unsigned)w2.y, (unsigned)w2.z};
                 TPhase ph[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) ph[k] = t_phase(t0, r0, d, k);
-                const int ngroups = t_shape_colgroups(shape);
-                const uint32_t box_bytes = (uint32_t)box_rows * kTBoxCols * 4u;
-                const uint32_t phase_bytes = (uint32_t)t_phase_floats(box_rows) * 4u;
-                const char* tmap = reinterpret_cast<const char*>(a.plan.tmaps) + (size_t)(2 * tk + shape) * 128;
+                const int nbx = t_boxes_per_phase(cg);
+                const uint32_t box_bytes = (uint32_t)box_rows * (uint32_t)t_box_cols(cg) * 4u;
+                const uint32_t phase_bytes = (uint32_t)t_phase_floats(cg, box_rows) * 4u;
+                const char* tmap = reinterpret_cast<const char*>(a.plan.tmaps) + (size_t)map * 128;
                 TParams* ps = params + (it % kTParamSlots);
                 for (int q = 0; q < m; ++q) {
                     const uint32_t slot = st % kTStages;
@@ -375,7 +389,7 @@ __global__ void __launch_bounds__(kTThreads, 4) fast_t_forward(FwdArgs a) {
                         break;
                     }
                     const uint32_t bar = full0 + 8u * slot;
-                    uint32_t tx = (uint32_t)ngroups * 4u * box_bytes;
+                    uint32_t tx = (uint32_t)nbx * 4u * box_bytes;
                     if (q == 0) tx += (uint32_t)sizeof(TParams);
                     mbar_arrive_expect_tx(bar, tx);
                     if (q == 0) {
@@ -385,10 +399,10 @@ __global__ void __launch_bounds__(kTThreads, 4) fast_t_forward(FwdArgs a) {
                     const int ch = (int)((chw[q >> 2] >> (8 * (q & 3))) & 0xffu);
                     const int z = n * a.C + ch;
                     const uint32_t dst0 = smem_u32(stages + slot * kTStageFloats);
-                    for (int wc = 0; wc < ngroups; ++wc)
+                    for (int bx = 0; bx < nbx; ++bx)
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            tma_load_3d(dst0 + (uint32_t)(wc * 4 + k) * phase_bytes, tmap, ph[k].x + kWarpCols * wc,
+                            tma_load_3d(dst0 + (uint32_t)(bx * 4 + k) * phase_bytes, tmap, ph[k].x + 2 * kWarpCols * bx,
                                         ph[k].y, z, bar);
                     ++st;
                 }
@@ -419,11 +433,12 @@ __global__ void __launch_bounds__(kTThreads, 4) fast_t_forward(FwdArgs a) {
             }
             const TParams* ps = params + (it % kTParamSlots);
             const KRec* rec = &ps->rec;
-            const int t0 = ps->item.t0, r0 = ps->item.r0, shape = ps->item.shape, box_rows = ps->item.box_rows;
+            const int t0 = ps->item.t0, r0 = ps->item.r0, rg = ps->item.rg, cg = ps->item.cg, box_rows = ps->item.box_rows;
             const int len = rec->len, d = rec->d, korig = rec->k, lo_u = rec->lo_u, hi_u = rec->hi_u;
-            const int wr = shape == 0 ? warp : (warp >> 1), wc = shape == 0 ? 0 : (warp & 1);
+            const int wr = cg == 1 ? warp : (cg == 2 ? warp >> 1 : warp >> 2), wc = warp & (cg - 1);
             const int lc = kWarpCols * wc + 2 * lane;
-            const bool ok0 = r0 + lc < d, ok1 = r0 + lc + 1 < d;
+            const bool in_tile = wr < rg;
+            const bool ok0 = in_tile && r0 + lc < d, ok1 = in_tile && r0 + lc + 1 < d;
             const int u00 = (t0 + kR * wr) * d + r0 + lc, u01 = u00 + 1;
             const bool mine = ok0 && ok1 && u00 >= lo_u && (u01 + (kR - 1) * d) < hi_u;
             const bool interior = __all_sync(kFull, mine);
@@ -432,26 +447,27 @@ __global__ void __launch_bounds__(kTThreads, 4) fast_t_forward(FwdArgs a) {
                 valid_rows(u00, d, lo_u, hi_u, kR, ok0, lo0, hi0);
                 valid_rows(u01, d, lo_u, hi_u, kR, ok1, lo1, hi1);
             }
+            const bool active = __any_sync(kFull, lo0 < hi0 || lo1 < hi1);
+            const int bx = cg == 1 ? 0 : wc >> 1, incol = cg == 1 ? 0 : (wc & 1) * kWarpCols;
+            const int boxw = t_box_cols(cg);
             int off[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-                off[k] = t_box_offset(wc, k, box_rows) + 4 * wr * kTBoxCols + (((t0 + k) * d) & 3) + 2 * lane;
+                off[k] = t_box_offset(cg, bx, k, box_rows) + 4 * wr * boxw + (((t0 + k) * d) & 3) + incol + 2 * lane;
             u64 acc[kR];
             const u64 negb = pack2(rec->negb, rec->negb);
 #pragma unroll
             for (int o = 0; o < kR; ++o) acc[o] = negb;
             const bool odd = (d & 1) != 0;
-            if (len == 7) ok = odd ? t_channels<7, true>(stages, rec, off, full0, empty0, st, lane, acc)
-                                   : t_channels<7, false>(stages, rec, off, full0, empty0, st, lane, acc);
-            else if (len == 9) ok = odd ? t_channels<9, true>(stages, rec, off, full0, empty0, st, lane, acc)
-                                        : t_channels<9, false>(stages, rec, off, full0, empty0, st, lane, acc);
-            else ok = odd ? t_channels<11, true>(stages, rec, off, full0, empty0, st, lane, acc)
-                          : t_channels<11, false>(stages, rec, off, full0, empty0, st, lane, acc);
+            if (cg == 1) ok = t_dispatch<kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
+            else ok = t_dispatch<2 * kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
             if (!ok) break;
-            int cnt = 0;
-            float mn = __int_as_float(0x7f800000);
-            pool_hard(acc, interior, lo0, hi0, lo1, hi1, cnt, mn);
-            publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
+            if (active) {
+                int cnt = 0;
+                float mn = __int_as_float(0x7f800000);
+                pool_hard(acc, interior, lo0, hi0, lo1, hi1, cnt, mn);
+                publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
+            }
             ++it;
         }
         if (!ok) {
@@ -542,7 +558,7 @@ cudaError_t upload_plan(FastState& fs) {
     d.counters = reinterpret_cast<unsigned*>(base + parts[5].off);
     d.error_flag = reinterpret_cast<int*>(base + parts[6].off);
     d.n_krec = (int)h.krec.size(); d.n_sitems = (int)h.sitems.size(); d.n_titems = (int)h.titems.size();
-    d.n_generic = (int)h.generic_list.size(); d.n_tkernels = (int)h.tkernels.size();
+    d.n_generic = (int)h.generic_list.size(); d.n_tmaps = (int)h.tmaps.size();
     d.pad_pitch = h.pad_pitch;
     return cudaSuccess;
 }
@@ -557,7 +573,7 @@ void release_fast_state(FastState& fs) {
 }
 
 cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L) {
-    if (fs.host.tkernels.empty() || N <= fs.pad_examples) return cudaSuccess;
+    if (fs.host.tmaps.empty() || N <= fs.pad_examples) return cudaSuccess;
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
     const int64_t pitch = fs.host.pad_pitch, rows = (int64_t)N * C;
@@ -569,22 +585,19 @@ cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L) {
     if (e != cudaSuccess) { fs.xpad = nullptr; return e; }
     e = cudaMemset(fs.xpad, 0, bytes);  // the margins stay zero from here on: the pad copy writes samples only
     if (e != cudaSuccess) return e;
-    const size_t n_maps = 2 * fs.host.tkernels.size();
+    const size_t n_maps = fs.host.tmaps.size();
     std::vector<CUtensorMap> maps(n_maps);
-    for (size_t i = 0; i < fs.host.tkernels.size(); ++i) {
-        const KRec& f = fs.host.krec[fs.host.tkernels[i]];
-        for (int shape = 0; shape < 2; ++shape) {
-            const cuuint64_t run = 4ull * (cuuint64_t)f.d;
-            const cuuint64_t dims[3] = {run + kTXExtra, ((cuuint64_t)kTPadFront + (cuuint64_t)L + run - 1) / run,
-                                        (cuuint64_t)rows};
-            const cuuint64_t strides[2] = {run * 4ull, (cuuint64_t)pitch * 4ull};
-            const cuuint32_t box[3] = {(cuuint32_t)kTBoxCols, (cuuint32_t)t_box_rows(shape, f.len), 1u};
-            const cuuint32_t elem[3] = {1u, 1u, 1u};
-            const CUresult r = encode(&maps[2 * i + shape], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, fs.xpad, dims, strides, box,
-                                      elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                                      CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-            if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
-        }
+    for (size_t i = 0; i < n_maps; ++i) {
+        const TMapSpec& sp = fs.host.tmaps[i];
+        const cuuint64_t run = 4ull * (cuuint64_t)sp.d;
+        const cuuint64_t dims[3] = {run + kTXExtra, ((cuuint64_t)kTPadFront + (cuuint64_t)L + run - 1) / run, (cuuint64_t)rows};
+        const cuuint64_t strides[2] = {run * 4ull, (cuuint64_t)pitch * 4ull};
+        const cuuint32_t box[3] = {(cuuint32_t)sp.box_cols, (cuuint32_t)sp.box_rows, 1u};
+        const cuuint32_t elem[3] = {1u, 1u, 1u};
+        const CUresult r = encode(&maps[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, fs.xpad, dims, strides, box, elem,
+                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
     static_assert(sizeof(CUtensorMap) == 128, "tensor maps are addressed in 128-byte steps");
     if (!fs.maps_blob) {
@@ -642,7 +655,7 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
     }
     if (pd.n_titems > 0) {
         const unsigned long long total = (unsigned long long)N * pd.n_titems;
-        const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms * 4);
+        const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms * 2);
         fast_t_forward<<<grid, kTThreads, t_bytes, stream>>>(a);
         count_launch();
     }

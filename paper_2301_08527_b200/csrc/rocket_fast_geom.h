@@ -52,12 +52,14 @@ ROCKET_HD TPhase t_phase(int t0, int r0, int d, int k) {
     return p;
 }
 
-// Float offset, inside a stage, of the box of column group wc and phase k.
-ROCKET_HD int t_box_offset(int wc, int k, int box_rows) { return (wc * 4 + k) * t_phase_floats(box_rows); }
+// Float offset, inside a stage, of box bx (0 or 1) of phase k.
+ROCKET_HD int t_box_offset(int cg, int bx, int k, int box_rows) { return (bx * 4 + k) * t_phase_floats(cg, box_rows); }
 
 // Float offset, inside a stage, of tile row s / tile column lc as the consumer reads it.
-ROCKET_HD int t_elem_offset(int s, int lc, int box_rows, int shift) {
-    return t_box_offset(lc >> 6, s & 3, box_rows) + (s >> 2) * kTBoxCols + shift + (lc & 63);
+ROCKET_HD int t_elem_offset(int cg, int s, int lc, int box_rows, int shift) {
+    const int wc = lc >> 6;
+    const int bx = cg == 1 ? 0 : wc >> 1, incol = cg == 1 ? 0 : (wc & 1) * kWarpCols;
+    return t_box_offset(cg, bx, s & 3, box_rows) + (s >> 2) * t_box_cols(cg) + shift + incol + (lc & 63);
 }
 
 }  // namespace fast

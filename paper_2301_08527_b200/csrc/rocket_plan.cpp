@@ -2,6 +2,7 @@
 // cuts them into tiles and orders the tiles by cost (largest first).
 #include <algorithm>
 #include <map>
+#include <tuple>
 
 #include "rocket_fast.h"
 
@@ -91,37 +92,61 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         out.sitems.swap(sorted);
     }
 
-    // ---- T regime: per kernel, bands of 64 rows (shape 0) and a last band of 32 (shape 1) or 64
+    // ---- T regime: per kernel, the grid of 16-row x 64-column warp tiles is cut into block tiles of
+    // rg x cg warp tiles (rg * cg <= 8); the column-group width that needs the fewest block tiles wins
     std::vector<Cost> t_cost;
     int d_max = 0;
+    std::map<std::tuple<int, int, int>, int> map_index;
     for (int k : t_kernels) {
         const int ki = (int)out.krec.size();
         add_kernel(k);
         const KRec f = out.krec.back();
-        const int tk = (int)out.tkernels.size();
-        out.tkernels.push_back(ki);
         d_max = std::max(d_max, f.d);
         int64_t tmin = floor_div(f.lo_u, f.d);
         const int64_t tmax = floor_div((int64_t)f.hi_u - 1, f.d);
         // odd dilations: an even first row keeps the rows of phases 0 and 2 aligned to pairs
         if (f.d & 1) tmin = floor_div(tmin, 2) * 2;
-        const int64_t rows = tmax - tmin + 1;
-        auto add_band = [&](int64_t t0, int shape) {
-            const int cols = kWarpCols * t_shape_colgroups(shape);
-            for (int r0 = 0; r0 < f.d; r0 += cols) {
+        const int R16 = (int)((tmax - tmin + 1 + kR - 1) / kR), C64 = (f.d + kWarpCols - 1) / kWarpCols;
+        // column chunks for a main width cg: C64 / cg chunks of cg, the rest in chunks of 2 and 1
+        auto chunks_of = [&](int cg, std::vector<int>& widths) {
+            widths.assign(C64 / cg, cg);
+            int rest = C64 % cg;
+            if (rest >= 2) { widths.push_back(2); rest -= 2; }
+            if (rest >= 1) widths.push_back(1);
+        };
+        int best_cg = 2;
+        int64_t best_tiles = INT64_MAX;
+        for (int cg : {2, 4, 1}) {
+            std::vector<int> widths;
+            chunks_of(cg, widths);
+            int64_t tiles = 0;
+            for (int w : widths) tiles += (R16 + 8 / w - 1) / (8 / w);
+            if (tiles < best_tiles) { best_tiles = tiles; best_cg = cg; }
+        }
+        std::vector<int> widths;
+        chunks_of(best_cg, widths);
+        int c64 = 0;
+        for (int w : widths) {
+            const int rg_full = 8 / w;
+            for (int r16 = 0; r16 < R16; r16 += rg_full) {
                 TItem it{};
-                it.tk = tk; it.t0 = (int32_t)t0; it.r0 = r0; it.shape = shape;
-                it.d = f.d; it.len = f.len; it.m = f.m; it.box_rows = t_box_rows(shape, f.len);
+                it.rg = std::min(rg_full, R16 - r16); it.cg = w;
+                it.t0 = (int32_t)(tmin + (int64_t)kR * r16); it.r0 = c64 * kWarpCols;
+                it.d = f.d; it.len = f.len; it.m = f.m; it.box_rows = t_box_rows(it.rg, f.len);
                 for (int q = 0; q < f.m; ++q) it.ch[q] = (uint8_t)f.ch[q];
                 it.krec = ki;
+                const auto key = std::make_tuple(f.d, t_box_cols(w), it.box_rows);
+                auto found = map_index.find(key);
+                if (found == map_index.end()) {
+                    found = map_index.emplace(key, (int)out.tmaps.size()).first;
+                    out.tmaps.push_back({f.d, t_box_cols(w), it.box_rows});
+                }
+                it.map = found->second;
                 t_cost.push_back({(double)f.m * (f.len + 2) + 6.0, (int)out.titems.size()});
                 out.titems.push_back(it);
             }
-        };
-        const int64_t full = rows / 64, rem = rows % 64;
-        for (int64_t b = 0; b < full; ++b) add_band(tmin + 64 * b, 0);
-        if (rem > 32) add_band(tmin + 64 * full, 0);
-        else if (rem > 0) add_band(tmin + 64 * full, 1);
+            c64 += w;
+        }
     }
     {
         std::stable_sort(t_cost.begin(), t_cost.end(), [](const Cost& a, const Cost& b) { return a.c > b.c; });
@@ -132,7 +157,7 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
     }
     // every channel row of the zero-margined copy: front zeros, L samples, zeros for the run a box may
     // read past the last sample; rounded to 128 bytes
-    const int64_t pitch = (int64_t)kTPadFront + hp.L + 4ll * d_max + kTXExtra + kTBoxCols;
+    const int64_t pitch = (int64_t)kTPadFront + hp.L + 4ll * d_max + kTXExtra + t_box_cols(2);
     out.pad_pitch = (pitch + 31) / 32 * 32;
 }
 

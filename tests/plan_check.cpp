@@ -79,30 +79,33 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
     REQUIRE(plan.titems.empty() || (pitch % 32 == 0 && pitch >= kTPadFront + L), "pad pitch");
     for (const TItem& it : plan.titems) {
         const KRec& f = plan.krec[it.krec];
-        REQUIRE(plan.tkernels[it.tk] == it.krec, "T kernel index");
+        REQUIRE(it.map >= 0 && it.map < (int)plan.tmaps.size(), "T map index");
+        const TMapSpec& sp = plan.tmaps[it.map];
         REQUIRE(f.d >= kTMinDilation && f.d == it.d && f.len == it.len && f.m == it.m, "T item fields");
-        REQUIRE(it.shape == 0 || it.shape == 1, "T shape");
+        REQUIRE((it.cg == 1 || it.cg == 2 || it.cg == 4) && it.rg >= 1 && it.rg * it.cg <= kTConsumerWarps, "T shape");
         REQUIRE(it.r0 % kWarpCols == 0 && it.r0 < f.d, "T column origin");
         REQUIRE(!(f.d & 1) || (it.t0 % 2 == 0), "odd dilation needs an even first row");
         for (int q = 0; q < f.m; ++q) REQUIRE(it.ch[q] == f.ch[q], "T channel list");
-        const int rows_out = t_shape_rows(it.shape), groups = t_shape_colgroups(it.shape);
+        const int rows_out = kR * it.rg, groups = it.cg, boxw = t_box_cols(it.cg), nbx = t_boxes_per_phase(it.cg);
         const int rows = rows_out + f.len - 1;
-        REQUIRE(it.box_rows == t_box_rows(it.shape, f.len) && 4 * it.box_rows >= rows, "T box rows");
+        REQUIRE(it.box_rows == t_box_rows(it.rg, f.len) && 4 * it.box_rows >= rows, "T box rows");
+        REQUIRE(sp.d == f.d && sp.box_cols == boxw && sp.box_rows == it.box_rows && boxw <= 256 && it.box_rows <= 256, "T map spec");
+        REQUIRE(4 * nbx * t_phase_floats(it.cg, it.box_rows) <= kTStageFloats, "stage size");
         const long long run = 4ll * f.d, ny = (kTPadFront + (long long)L + run - 1) / run;
         // the boxes the producer issues
         TPhase ph[4];
         for (int k = 0; k < 4; ++k) {
             ph[k] = t_phase(it.t0, it.r0, f.d, k);
             REQUIRE(ph[k].x % 4 == 0 && ph[k].x >= 0 && ph[k].x < run, "box x");
-            for (int wc = 0; wc < groups; ++wc) {
-                const int x = ph[k].x + kWarpCols * wc;
-                REQUIRE(x + kTBoxCols <= run + kTXExtra, "box leaves the tensor row");
-                const int dst = t_box_offset(wc, k, it.box_rows);
-                REQUIRE(dst % 32 == 0 && dst + it.box_rows * kTBoxCols <= kTStageFloats, "box destination");
+            for (int bx = 0; bx < nbx; ++bx) {
+                const int x = ph[k].x + 2 * kWarpCols * bx;
+                REQUIRE(x + boxw <= run + kTXExtra, "box leaves the tensor row");
+                const int dst = t_box_offset(it.cg, bx, k, it.box_rows);
+                REQUIRE(dst % 32 == 0 && dst + it.box_rows * boxw <= kTStageFloats, "box destination");
                 for (int j = 0; j < it.box_rows; ++j) {
                     const long long y = ph[k].y + j;
                     if (y < 0 || y >= ny) continue;  // zero-filled by the copy engine
-                    const long long first = y * run + x, last = first + kTBoxCols - 1;
+                    const long long first = y * run + x, last = first + boxw - 1;
                     REQUIRE(first >= 0 && last < pitch, "box row reads outside its channel row: %lld..%lld of %lld", first,
                             last, (long long)pitch);
                 }
@@ -111,7 +114,7 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
         // what every consumer thread owns and reads
         for (int lc = 0; lc < kWarpCols * groups; ++lc) {
             const bool col_ok = it.r0 + lc < f.d;
-            for (int wr = 0; wr < rows_out / kR; ++wr) {
+            for (int wr = 0; wr < it.rg; ++wr) {
                 const int u0 = (it.t0 + kR * wr) * f.d + it.r0 + lc;
                 int o_lo, o_hi;
                 valid_rows(u0, f.d, f.lo_u, f.hi_u, kR, col_ok, o_lo, o_hi);
@@ -125,16 +128,16 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
                     const int s = kR * wr + s2, k = s & 3;
                     const int shift = ((it.t0 + k) * f.d) & 3;
                     REQUIRE(shift == ph[k].shift, "alignment shift");
-                    const int pos = t_elem_offset(s, lc, it.box_rows, shift);
+                    const int pos = t_elem_offset(it.cg, s, lc, it.box_rows, shift);
                     REQUIRE(pos >= 0 && pos < kTStageFloats, "read outside the stage");
                     if ((lc & 1) == 0) REQUIRE(((f.d & 1) && (s2 & 1)) || pos % 2 == 0, "pair not 8-byte aligned");
                     // which sample the copy engine put there
-                    const int wc = lc >> 6;
-                    const int rel = pos - t_box_offset(wc, k, it.box_rows);
-                    const int j = rel / kTBoxCols, i = rel % kTBoxCols;
-                    REQUIRE(j < it.box_rows, "read below the box");
+                    const int wc = lc >> 6, bx = it.cg == 1 ? 0 : wc >> 1;
+                    const int rel = pos - t_box_offset(it.cg, bx, k, it.box_rows);
+                    const int j = rel / boxw, i = rel % boxw;
+                    REQUIRE(rel >= 0 && j < it.box_rows, "read outside the box");
                     const long long y = ph[k].y + j;
-                    const long long flat = y * run + ph[k].x + kWarpCols * wc + i;
+                    const long long flat = y * run + ph[k].x + 2 * kWarpCols * bx + i;
                     const long long want = (long long)kTPadFront + (long long)(it.t0 + s) * f.d + it.r0 + lc;
                     REQUIRE(flat == want, "wrong sample: got flat %lld, want %lld", flat, want);
                     const bool in_series = want >= kTPadFront && want < kTPadFront + L;
