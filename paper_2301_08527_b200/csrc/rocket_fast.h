@@ -93,15 +93,17 @@ constexpr int kTStageFloats = imax_cx(imax_cx(t_stage_floats(8, 1, ROCKET_MAX_LE
 constexpr int kTPadFront = 128;                                    // zero floats before every channel row
 constexpr int kTXExtra = 256;                                      // floats a box may run past a 4d run
 
-// One T tile with everything the producer warp needs (16 words).
+// One T tile with everything the producer warp needs (32 words).
 struct alignas(16) TItem {
     int32_t map, t0, r0, rg;              // map: index of the tile's tensor map; tile origin (t0, r0)
     int32_t d, len, m, box_rows;
     uint8_t ch[12];
     int32_t krec;                         // index into the kernel records
-    int32_t cg, pad_[3];
+    int32_t cg, pad0_[3];
+    int32_t x[4], y[4];                   // tensor coordinates of the four phase boxes
+    int32_t pad1_[8];
 };
-static_assert(sizeof(TItem) == 64, "TItem must be 16 words");
+static_assert(sizeof(TItem) == 128, "TItem must be 32 words");
 // One tensor map: boxes of box_cols x box_rows floats over runs of 4 * d floats.
 struct TMapSpec { int32_t d, box_cols, box_rows; };
 
@@ -111,7 +113,8 @@ struct PlanHost {
     std::vector<KRec> krec;
     std::vector<SBucket> sb;
     std::vector<SItem> sitems;
-    std::vector<TItem> titems;
+    std::vector<TItem> titems;            // kernel by kernel, in the order the blocks walk them
+    std::vector<double> tcost;            // relative cost of every T tile
     std::vector<TMapSpec> tmaps;          // tensor maps the T tiles refer to
     std::vector<int32_t> generic_list;    // kernels the fast path does not take
     int64_t pad_pitch = 0;                // floats per channel row of the zero-margined copy
@@ -122,13 +125,14 @@ struct PlanDevice {
     const SBucket* sb = nullptr;
     const SItem* sitems = nullptr;
     const TItem* titems = nullptr;
+    const int32_t* tranges = nullptr;     // [n_tblocks + 1]: block b walks T tiles [tranges[b], tranges[b+1]) of every example
     const int32_t* generic_list = nullptr;
     unsigned* counters = nullptr;         // [0] S work counter
     int* error_flag = nullptr;            // set when a bounded wait gave up
     const void* tmaps = nullptr;          // CUtensorMap[n_tmaps], 128 bytes each
     float* xpad = nullptr;                // zero-margined copy of the batch
     int64_t pad_pitch = 0;
-    int n_krec = 0, n_sitems = 0, n_titems = 0, n_generic = 0, n_tmaps = 0;
+    int n_krec = 0, n_sitems = 0, n_titems = 0, n_generic = 0, n_tmaps = 0, n_tblocks = 0;
 };
 
 // Builds the launch plan for the kernels in hp (host side, once per handle).

@@ -295,15 +295,16 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, int 
         ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
 
-struct TParams {
-    KRec rec;
-    TItem item;
+// What the producer tells the consumers about a tile (written with plain stores before its
+// arrive on the stage's barrier, which releases them).
+struct TSlotItem {
+    int32_t t0, r0, rg, cg, box_rows, rec_slot, pad_[2];
 };
-static_assert(sizeof(TParams) % 16 == 0, "parameter slots must stay 16-byte aligned");
 
 struct TShared {
     unsigned long long full[kTStages];
     unsigned long long empty[kTStages];
+    TSlotItem items[kTParamSlots];
     int abort;
 };
 
@@ -337,12 +338,12 @@ __device__ __forceinline__ bool t_dispatch(int len, bool odd, const float* stage
 }
 
 __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
-    __shared__ __align__(8) TShared sh;
-    // dynamic shared memory, aligned to 128 bytes by hand: stages, then parameter slots
+    __shared__ __align__(16) TShared sh;
+    // dynamic shared memory, aligned to 128 bytes by hand: stages, then kernel-record slots
     const uint32_t raw = smem_u32(smem_raw);
     unsigned char* base = smem_raw + (((raw + 127u) & ~127u) - raw);
     float* stages = reinterpret_cast<float*>(base);
-    TParams* params = reinterpret_cast<TParams*>(base + (size_t)kTStages * kTStageFloats * 4);
+    KRec* recs = reinterpret_cast<KRec*>(base + (size_t)kTStages * kTStageFloats * 4);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t full0 = smem_u32(sh.full), empty0 = smem_u32(sh.empty);
     if (threadIdx.x == 0) {
@@ -354,59 +355,68 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    const unsigned n_items = (unsigned)a.plan.n_titems;
-    const unsigned long long total = (unsigned long long)a.N * n_items;
+    // every block walks the same slice of the tile list for every example in turn, so that all
+    // blocks read one example at a time (it stays in L2) and consecutive tiles share a kernel
+    const int i_beg = a.plan.tranges[blockIdx.x], i_end = a.plan.tranges[blockIdx.x + 1];
     volatile int* abort_flag = &sh.abort;
 
     if (warp == kTConsumerWarps) {
         // ---- producer: one lane issues every copy of the block
-        if (lane == 0) {
-            uint32_t st = 0, it = 0;
+        if (lane == 0 && i_beg < i_end) {
+            uint32_t st = 0, it = 0, nrec = 0;
+            int cur_krec = -1;
             bool ok = true;
-            for (unsigned long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
-                if (*abort_flag) break;
-                const int n = (int)(g / n_items);
-                const TItem* tp = a.plan.titems + (g - (unsigned long long)n * n_items);
-                const int4 w0 = __ldg(reinterpret_cast<const int4*>(tp));
-                const int4 w1 = __ldg(reinterpret_cast<const int4*>(tp) + 1);
-                const int4 w2 = __ldg(reinterpret_cast<const int4*>(tp) + 2);
-                const int cg = __ldg(reinterpret_cast<const int*>(tp) + 12);
-                const int map = w0.x, t0 = w0.y, r0 = w0.z;
-                const int d = w1.x, m = w1.z, box_rows = w1.w;
-                const unsigned chw[3] = {(unsigned)w2.x, (unsigned)w2.y, (unsigned)w2.z};
-                TPhase ph[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) ph[k] = t_phase(t0, r0, d, k);
-                const int nbx = t_boxes_per_phase(cg);
-                const uint32_t box_bytes = (uint32_t)box_rows * (uint32_t)t_box_cols(cg) * 4u;
-                const uint32_t phase_bytes = (uint32_t)t_phase_floats(cg, box_rows) * 4u;
-                const char* tmap = reinterpret_cast<const char*>(a.plan.tmaps) + (size_t)map * 128;
-                TParams* ps = params + (it % kTParamSlots);
-                for (int q = 0; q < m; ++q) {
-                    const uint32_t slot = st % kTStages;
-                    if (st >= (uint32_t)kTStages && !mbar_wait(empty0 + 8u * slot, ((st / kTStages) - 1u) & 1u)) {
-                        ok = false;
-                        break;
+            const int4* tp = reinterpret_cast<const int4*>(a.plan.titems + i_beg);
+            int4 w0 = __ldg(tp), w1 = __ldg(tp + 1), w2 = __ldg(tp + 2), w3 = __ldg(tp + 3), w4 = __ldg(tp + 4),
+                 w5 = __ldg(tp + 5);
+            for (int n = 0; ok && n < a.N; ++n) {
+                for (int i = i_beg; ok && i < i_end; ++i) {
+                    if (*abort_flag) { ok = false; break; }
+                    const int map = w0.x, t0 = w0.y, r0 = w0.z, rg = w0.w;
+                    const int m = w1.z, box_rows = w1.w, krec = w2.w, cg = w3.x;
+                    const unsigned chw[3] = {(unsigned)w2.x, (unsigned)w2.y, (unsigned)w2.z};
+                    const int px[4] = {w4.x, w4.y, w4.z, w4.w}, py[4] = {w5.x, w5.y, w5.z, w5.w};
+                    {   // the next tile's description is on its way while this one is issued
+                        int inext = i + 1;
+                        if (inext == i_end) inext = i_beg;
+                        tp = reinterpret_cast<const int4*>(a.plan.titems + inext);
+                        w0 = __ldg(tp); w1 = __ldg(tp + 1); w2 = __ldg(tp + 2); w3 = __ldg(tp + 3); w4 = __ldg(tp + 4);
+                        w5 = __ldg(tp + 5);
                     }
-                    const uint32_t bar = full0 + 8u * slot;
-                    uint32_t tx = (uint32_t)nbx * 4u * box_bytes;
-                    if (q == 0) tx += (uint32_t)sizeof(TParams);
-                    mbar_arrive_expect_tx(bar, tx);
-                    if (q == 0) {
-                        bulk_g2s(smem_u32(&ps->rec), a.plan.krec + w2.w, (uint32_t)sizeof(KRec), bar);
-                        bulk_g2s(smem_u32(&ps->item), tp, (uint32_t)sizeof(TItem), bar);
-                    }
-                    const int ch = (int)((chw[q >> 2] >> (8 * (q & 3))) & 0xffu);
-                    const int z = n * a.C + ch;
-                    const uint32_t dst0 = smem_u32(stages + slot * kTStageFloats);
-                    for (int bx = 0; bx < nbx; ++bx)
+                    const int nbx = t_boxes_per_phase(cg);
+                    const uint32_t box_bytes = (uint32_t)box_rows * (uint32_t)t_box_cols(cg) * 4u;
+                    const uint32_t phase_bytes = (uint32_t)t_phase_floats(cg, box_rows) * 4u;
+                    const char* tmap = reinterpret_cast<const char*>(a.plan.tmaps) + (size_t)map * 128;
+                    const bool new_rec = krec != cur_krec;
+                    if (new_rec) { cur_krec = krec; ++nrec; }
+                    const uint32_t rslot = (nrec - 1u) % kTParamSlots;
+                    for (int q = 0; q < m; ++q) {
+                        const uint32_t slot = st % kTStages;
+                        if (st >= (uint32_t)kTStages && !mbar_wait(empty0 + 8u * slot, ((st / kTStages) - 1u) & 1u)) {
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t bar = full0 + 8u * slot;
+                        uint32_t tx = (uint32_t)nbx * 4u * box_bytes;
+                        if (q == 0) {
+                            TSlotItem& si = sh.items[it % kTParamSlots];
+                            si.t0 = t0; si.r0 = r0; si.rg = rg; si.cg = cg; si.box_rows = box_rows; si.rec_slot = (int)rslot;
+                            if (new_rec) tx += (uint32_t)sizeof(KRec);
+                        }
+                        mbar_arrive_expect_tx(bar, tx);
+                        if (q == 0 && new_rec) bulk_g2s(smem_u32(recs + rslot), a.plan.krec + krec, (uint32_t)sizeof(KRec), bar);
+                        const int ch = (int)((chw[q >> 2] >> (8 * (q & 3))) & 0xffu);
+                        const int z = n * a.C + ch;
+                        const uint32_t dst0 = smem_u32(stages + slot * kTStageFloats);
+                        for (int bx = 0; bx < nbx; ++bx)
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            tma_load_3d(dst0 + (uint32_t)(bx * 4 + k) * phase_bytes, tmap, ph[k].x + 2 * kWarpCols * bx,
-                                        ph[k].y, z, bar);
-                    ++st;
+                            for (int k = 0; k < 4; ++k)
+                                tma_load_3d(dst0 + (uint32_t)(bx * 4 + k) * phase_bytes, tmap, px[k] + 2 * kWarpCols * bx, py[k], z,
+                                            bar);
+                        ++st;
+                    }
+                    ++it;
                 }
-                ++it;
             }
             if (!ok) {
                 *abort_flag = 1;
@@ -423,52 +433,53 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
         // ---- consumers
         uint32_t st = 0, it = 0;
         bool ok = true;
-        for (unsigned long long g = blockIdx.x; ok && g < total; g += gridDim.x) {
-            if (*abort_flag) break;
-            const int n = (int)(g / n_items);
-            const uint32_t slot = st % kTStages;
-            if (!mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) {
-                ok = false;
-                break;
-            }
-            const TParams* ps = params + (it % kTParamSlots);
-            const KRec* rec = &ps->rec;
-            const int t0 = ps->item.t0, r0 = ps->item.r0, rg = ps->item.rg, cg = ps->item.cg, box_rows = ps->item.box_rows;
-            const int len = rec->len, d = rec->d, korig = rec->k, lo_u = rec->lo_u, hi_u = rec->hi_u;
-            const int wr = cg == 1 ? warp : (cg == 2 ? warp >> 1 : warp >> 2), wc = warp & (cg - 1);
-            const int lc = kWarpCols * wc + 2 * lane;
-            const bool in_tile = wr < rg;
-            const bool ok0 = in_tile && r0 + lc < d, ok1 = in_tile && r0 + lc + 1 < d;
-            const int u00 = (t0 + kR * wr) * d + r0 + lc, u01 = u00 + 1;
-            const bool mine = ok0 && ok1 && u00 >= lo_u && (u01 + (kR - 1) * d) < hi_u;
-            const bool interior = __all_sync(kFull, mine);
-            int lo0 = 0, hi0 = kR, lo1 = 0, hi1 = kR;
-            if (!interior) {
-                valid_rows(u00, d, lo_u, hi_u, kR, ok0, lo0, hi0);
-                valid_rows(u01, d, lo_u, hi_u, kR, ok1, lo1, hi1);
-            }
-            const bool active = __any_sync(kFull, lo0 < hi0 || lo1 < hi1);
-            const int bx = cg == 1 ? 0 : wc >> 1, incol = cg == 1 ? 0 : (wc & 1) * kWarpCols;
-            const int boxw = t_box_cols(cg);
-            int off[4];
+        for (int n = 0; ok && n < a.N; ++n) {
+            for (int i = i_beg; ok && i < i_end; ++i) {
+                if (*abort_flag) { ok = false; break; }
+                const uint32_t slot = st % kTStages;
+                if (!mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) {
+                    ok = false;
+                    break;
+                }
+                const TSlotItem si = sh.items[it % kTParamSlots];
+                const KRec* rec = recs + si.rec_slot;
+                const int t0 = si.t0, r0 = si.r0, rg = si.rg, cg = si.cg, box_rows = si.box_rows;
+                const int len = rec->len, d = rec->d, korig = rec->k, lo_u = rec->lo_u, hi_u = rec->hi_u;
+                const int wr = cg == 1 ? warp : (cg == 2 ? warp >> 1 : warp >> 2), wc = warp & (cg - 1);
+                const int lc = kWarpCols * wc + 2 * lane;
+                const bool in_tile = wr < rg;
+                const bool ok0 = in_tile && r0 + lc < d, ok1 = in_tile && r0 + lc + 1 < d;
+                const int u00 = (t0 + kR * wr) * d + r0 + lc, u01 = u00 + 1;
+                const bool mine = ok0 && ok1 && u00 >= lo_u && (u01 + (kR - 1) * d) < hi_u;
+                const bool interior = __all_sync(kFull, mine);
+                int lo0 = 0, hi0 = kR, lo1 = 0, hi1 = kR;
+                if (!interior) {
+                    valid_rows(u00, d, lo_u, hi_u, kR, ok0, lo0, hi0);
+                    valid_rows(u01, d, lo_u, hi_u, kR, ok1, lo1, hi1);
+                }
+                const bool active = __any_sync(kFull, lo0 < hi0 || lo1 < hi1);
+                const int bx = cg == 1 ? 0 : wc >> 1, incol = cg == 1 ? 0 : (wc & 1) * kWarpCols;
+                const int boxw = t_box_cols(cg);
+                int off[4];
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                off[k] = t_box_offset(cg, bx, k, box_rows) + 4 * wr * boxw + (((t0 + k) * d) & 3) + incol + 2 * lane;
-            u64 acc[kR];
-            const u64 negb = pack2(rec->negb, rec->negb);
+                for (int k = 0; k < 4; ++k)
+                    off[k] = t_box_offset(cg, bx, k, box_rows) + 4 * wr * boxw + (((t0 + k) * d) & 3) + incol + 2 * lane;
+                u64 acc[kR];
+                const u64 negb = pack2(rec->negb, rec->negb);
 #pragma unroll
-            for (int o = 0; o < kR; ++o) acc[o] = negb;
-            const bool odd = (d & 1) != 0;
-            if (cg == 1) ok = t_dispatch<kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
-            else ok = t_dispatch<2 * kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
-            if (!ok) break;
-            if (active) {
-                int cnt = 0;
-                float mn = __int_as_float(0x7f800000);
-                pool_hard(acc, interior, lo0, hi0, lo1, hi1, cnt, mn);
-                publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
+                for (int o = 0; o < kR; ++o) acc[o] = negb;
+                const bool odd = (d & 1) != 0;
+                if (cg == 1) ok = t_dispatch<kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
+                else ok = t_dispatch<2 * kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
+                if (!ok) break;
+                if (active) {
+                    int cnt = 0;
+                    float mn = __int_as_float(0x7f800000);
+                    pool_hard(acc, interior, lo0, hi0, lo1, hi1, cnt, mn);
+                    publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
+                }
+                ++it;
             }
-            ++it;
         }
         if (!ok) {
             *abort_flag = 1;
@@ -512,7 +523,7 @@ __global__ void fast_finalize_kernel(float* __restrict__ feat, const KRec* __res
 size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 size_t s_smem_bytes(int C) { return (size_t)C * kSPlaneFloats * 4 + (size_t)kSWarps * 2 * sizeof(KRec); }
-size_t t_smem_bytes() { return (size_t)kTStages * kTStageFloats * 4 + (size_t)kTParamSlots * sizeof(TParams) + 128; }
+size_t t_smem_bytes() { return (size_t)kTStages * kTStageFloats * 4 + (size_t)kTParamSlots * sizeof(KRec) + 128; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -536,27 +547,48 @@ cudaError_t upload_plan(FastState& fs) {
     const PlanHost& h = fs.host;
     PlanDevice& d = fs.dev;
     d = PlanDevice();
+    // the T tile list is cut into one slice of equal cost per block (two blocks per SM)
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const int n_tblocks = h.titems.empty() ? 0 : (int)std::min<size_t>(h.titems.size(), (size_t)sms * 2);
+    std::vector<int32_t> tranges(n_tblocks + 1, 0);
+    if (n_tblocks > 0) {
+        double total_cost = 0.0;
+        for (double c : h.tcost) total_cost += c;
+        double run = 0.0;
+        int b = 1;
+        for (size_t i = 0; i < h.titems.size() && b < n_tblocks; ++i) {
+            run += h.tcost[i];
+            while (b < n_tblocks && run >= total_cost * b / n_tblocks) tranges[b++] = (int32_t)(i + 1);
+        }
+        for (; b <= n_tblocks; ++b) tranges[b] = (int32_t)h.titems.size();
+    }
     struct Part { const void* src; size_t bytes; size_t off; };
-    Part parts[7] = {
+    Part parts[8] = {
+        {tranges.data(), tranges.size() * 4, 0},
         {h.krec.data(), h.krec.size() * sizeof(KRec), 0},   {h.sb.data(), h.sb.size() * sizeof(SBucket), 0},
         {h.sitems.data(), h.sitems.size() * sizeof(SItem), 0}, {h.titems.data(), h.titems.size() * sizeof(TItem), 0},
         {h.generic_list.data(), h.generic_list.size() * 4, 0}, {nullptr, 256, 0}, {nullptr, 256, 0}};
     size_t total = 0;
     for (auto& pt : parts) { pt.off = total; total += align256(pt.bytes); }
-    cudaError_t e = cudaMalloc(&fs.plan_blob, std::max<size_t>(total, 256));
+    e = cudaMalloc(&fs.plan_blob, std::max<size_t>(total, 256));
     if (e != cudaSuccess) { fs.plan_blob = nullptr; return e; }
     char* base = static_cast<char*>(fs.plan_blob);
     e = cudaMemset(base, 0, std::max<size_t>(total, 256));
     for (auto& pt : parts)
         if (e == cudaSuccess && pt.src && pt.bytes) e = cudaMemcpy(base + pt.off, pt.src, pt.bytes, cudaMemcpyHostToDevice);
     if (e != cudaSuccess) { cudaFree(fs.plan_blob); fs.plan_blob = nullptr; return e; }
-    d.krec = reinterpret_cast<const KRec*>(base + parts[0].off);
-    d.sb = reinterpret_cast<const SBucket*>(base + parts[1].off);
-    d.sitems = reinterpret_cast<const SItem*>(base + parts[2].off);
-    d.titems = reinterpret_cast<const TItem*>(base + parts[3].off);
-    d.generic_list = reinterpret_cast<const int32_t*>(base + parts[4].off);
-    d.counters = reinterpret_cast<unsigned*>(base + parts[5].off);
-    d.error_flag = reinterpret_cast<int*>(base + parts[6].off);
+    d.krec = reinterpret_cast<const KRec*>(base + parts[1].off);
+    d.sb = reinterpret_cast<const SBucket*>(base + parts[2].off);
+    d.sitems = reinterpret_cast<const SItem*>(base + parts[3].off);
+    d.titems = reinterpret_cast<const TItem*>(base + parts[4].off);
+    d.generic_list = reinterpret_cast<const int32_t*>(base + parts[5].off);
+    d.counters = reinterpret_cast<unsigned*>(base + parts[6].off);
+    d.error_flag = reinterpret_cast<int*>(base + parts[7].off);
+    d.tranges = reinterpret_cast<const int32_t*>(base + parts[0].off);
+    d.n_tblocks = n_tblocks;
     d.n_krec = (int)h.krec.size(); d.n_sitems = (int)h.sitems.size(); d.n_titems = (int)h.titems.size();
     d.n_generic = (int)h.generic_list.size(); d.n_tmaps = (int)h.tmaps.size();
     d.pad_pitch = h.pad_pitch;
@@ -654,9 +686,7 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
         count_launch();
     }
     if (pd.n_titems > 0) {
-        const unsigned long long total = (unsigned long long)N * pd.n_titems;
-        const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms * 2);
-        fast_t_forward<<<grid, kTThreads, t_bytes, stream>>>(a);
+        fast_t_forward<<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
         count_launch();
     }
     const int64_t fin = (int64_t)N * pd.n_krec;

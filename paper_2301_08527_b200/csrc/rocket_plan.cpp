@@ -5,6 +5,7 @@
 #include <tuple>
 
 #include "rocket_fast.h"
+#include "rocket_fast_geom.h"
 
 namespace rocket {
 namespace fast {
@@ -94,7 +95,6 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
 
     // ---- T regime: per kernel, the grid of 16-row x 64-column warp tiles is cut into block tiles of
     // rg x cg warp tiles (rg * cg <= 8); the column-group width that needs the fewest block tiles wins
-    std::vector<Cost> t_cost;
     int d_max = 0;
     std::map<std::tuple<int, int, int>, int> map_index;
     for (int k : t_kernels) {
@@ -142,18 +142,15 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
                     out.tmaps.push_back({f.d, t_box_cols(w), it.box_rows});
                 }
                 it.map = found->second;
-                t_cost.push_back({(double)f.m * (f.len + 2) + 6.0, (int)out.titems.size()});
+                for (int ph = 0; ph < 4; ++ph) {
+                    const TPhase tp = t_phase(it.t0, it.r0, it.d, ph);
+                    it.x[ph] = tp.x; it.y[ph] = tp.y;
+                }
+                out.tcost.push_back((double)f.m * (f.len + 2) + 8.0);
                 out.titems.push_back(it);
             }
             c64 += w;
         }
-    }
-    {
-        std::stable_sort(t_cost.begin(), t_cost.end(), [](const Cost& a, const Cost& b) { return a.c > b.c; });
-        std::vector<TItem> sorted;
-        sorted.reserve(out.titems.size());
-        for (auto& c : t_cost) sorted.push_back(out.titems[c.idx]);
-        out.titems.swap(sorted);
     }
     // every channel row of the zero-margined copy: front zeros, L samples, zeros for the run a box may
     // read past the last sample; rounded to 128 bytes

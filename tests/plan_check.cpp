@@ -77,6 +77,7 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
 
     const int64_t pitch = plan.pad_pitch;
     REQUIRE(plan.titems.empty() || (pitch % 32 == 0 && pitch >= kTPadFront + L), "pad pitch");
+    REQUIRE(plan.tcost.size() == plan.titems.size(), "one cost per T tile");
     for (const TItem& it : plan.titems) {
         const KRec& f = plan.krec[it.krec];
         REQUIRE(it.map >= 0 && it.map < (int)plan.tmaps.size(), "T map index");
@@ -97,6 +98,7 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
         for (int k = 0; k < 4; ++k) {
             ph[k] = t_phase(it.t0, it.r0, f.d, k);
             REQUIRE(ph[k].x % 4 == 0 && ph[k].x >= 0 && ph[k].x < run, "box x");
+            REQUIRE(it.x[k] == ph[k].x && it.y[k] == ph[k].y, "stored box coordinates");
             for (int bx = 0; bx < nbx; ++bx) {
                 const int x = ph[k].x + 2 * kWarpCols * bx;
                 REQUIRE(x + boxw <= run + kTXExtra, "box leaves the tensor row");
