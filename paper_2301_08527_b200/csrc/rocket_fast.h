@@ -52,7 +52,8 @@ struct alignas(16) KRec {
     int32_t nout, k, lo_u, hi_u;   // k: original kernel index; lo_u = -p; hi_u = nout - p (exclusive)
     float negb;                    // 0 - bias (never -0.0)
     int32_t ch[ROCKET_MAX_CHANNELS_PER_KERNEL];
-    int32_t pad_[12];
+    int32_t tl, rl, th, rh;        // lo_u = tl * d + rl and hi_u = th * d + rh with 0 <= rl, rh < d
+    int32_t pad_[8];
     // w2[q][2j] = w2[q][2j+1] = 0 - W[q][j]: each weight twice, ready as a packed pair
     float w2[ROCKET_MAX_CHANNELS_PER_KERNEL][kPairRow];
 };

@@ -84,29 +84,32 @@ __device__ __forceinline__ void conv_channel(const float* __restrict__ st, const
     }
 }
 
-// PPV count and min(-z) over the thread's 2 x 16 outputs; rows outside [lo, hi) of either column
-// are neutralised.
-__device__ __forceinline__ void pool_hard(const u64 (&acc)[kR], bool interior, int lo0, int hi0, int lo1, int hi1,
-                                          int& cnt, float& mn) {
-    const float inf = __int_as_float(0x7f800000);
+// PPV count and min(-z) over the thread's 2 x 16 outputs.  Outputs outside the kernel's range
+// never need a test here: their accumulators start at +inf and stay there (sign bit clear,
+// neutral for the min).
+__device__ __forceinline__ void pool_hard(const u64 (&acc)[kR], int& cnt, float& mn) {
+    unsigned signs = 0;  // one sign bit per output, shifted in from the right
+#pragma unroll
+    for (int o = 0; o < kR; ++o) {
+        float a, b;
+        unpack2(acc[o], a, b);
+        signs = __funnelshift_l(__float_as_uint(a), signs, 1);
+        signs = __funnelshift_l(__float_as_uint(b), signs, 1);
+        mn = min3(mn, a, b);
+    }
+    cnt = __popc(signs);
+}
+
+// Accumulators of a tile: 0 - bias where the output exists, +inf elsewhere.
+__device__ __forceinline__ void init_acc(u64 (&acc)[kR], float negb, bool interior, int lo0, int hi0, int lo1, int hi1) {
     if (interior) {
+        const u64 v = pack2(negb, negb);
 #pragma unroll
-        for (int o = 0; o < kR; ++o) {
-            float a, b;
-            unpack2(acc[o], a, b);
-            cnt += (int)(__float_as_uint(a) >> 31) + (int)(__float_as_uint(b) >> 31);
-            mn = min3(mn, a, b);
-        }
+        for (int o = 0; o < kR; ++o) acc[o] = v;
     } else {
+        const float inf = __int_as_float(0x7f800000);
 #pragma unroll
-        for (int o = 0; o < kR; ++o) {
-            float a, b;
-            unpack2(acc[o], a, b);
-            if (o < lo0 || o >= hi0) a = inf;
-            if (o < lo1 || o >= hi1) b = inf;
-            cnt += (int)(__float_as_uint(a) >> 31) + (int)(__float_as_uint(b) >> 31);
-            mn = min3(mn, a, b);
-        }
+        for (int o = 0; o < kR; ++o) acc[o] = pack2((o >= lo0 && o < hi0) ? negb : inf, (o >= lo1 && o < hi1) ? negb : inf);
     }
 }
 
@@ -143,9 +146,6 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 
 template <int ELL>
 __device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* rec, int lane, u64 (&acc)[kR]) {
-    const u64 negb = pack2(rec->negb, rec->negb);
-#pragma unroll
-    for (int o = 0; o < kR; ++o) acc[o] = negb;
     const int m = rec->m;
     const int off[4] = {2 * lane, kWarpCols + 2 * lane, 2 * kWarpCols + 2 * lane, 3 * kWarpCols + 2 * lane};
     for (int q = 0; q < m; ++q)
@@ -197,7 +197,9 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
         // the thread's two columns
         const int cg0 = item.c0 + 2 * lane;
         const bool ok0 = cg0 < b.raster_len, ok1 = cg0 + 1 < b.raster_len;
-        const int u00 = s_column_u0(b, cg0), u01 = s_column_u0(b, cg0 + 1);
+        const int band0 = cg0 / d, c0 = cg0 - band0 * d;          // (first A-row, residue) of the two columns
+        const int band1 = c0 + 1 < d ? band0 : band0 + 1, c1 = c0 + 1 < d ? c0 + 1 : 0;
+        const int trow0 = b.tmin + band0 * kR, trow1 = b.tmin + band1 * kR;
         if (threadIdx.x == 0) s_next = b.kbeg;
         cp_async_wait<0>();
         __syncthreads();
@@ -225,22 +227,19 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
             cp_async_wait<1>();
             __syncwarp();
             const KRec* rec = myrec + cur;
-            const int len = rec->len, korig = rec->k, lo_u = rec->lo_u, hi_u = rec->hi_u;
-            const bool mine = ok0 && ok1 && u00 >= lo_u && u01 >= lo_u && (u00 + (kR - 1) * d) < hi_u &&
-                              (u01 + (kR - 1) * d) < hi_u;
-            const bool interior = __all_sync(kFull, mine);
-            int lo0 = 0, hi0 = kR, lo1 = 0, hi1 = kR;
-            if (!interior) {
-                valid_rows(u00, d, lo_u, hi_u, kR, ok0, lo0, hi0);
-                valid_rows(u01, d, lo_u, hi_u, kR, ok1, lo1, hi1);
-            }
+            const int len = rec->len, korig = rec->k;
+            int lo0, hi0, lo1, hi1;
+            valid_rows_tc(trow0, c0, rec->tl, rec->rl, rec->th, rec->rh, kR, ok0, lo0, hi0);
+            valid_rows_tc(trow1, c1, rec->tl, rec->rl, rec->th, rec->rh, kR, ok1, lo1, hi1);
+            const bool interior = __all_sync(kFull, lo0 == 0 && lo1 == 0 && hi0 == kR && hi1 == kR);
             u64 acc[kR];
+            init_acc(acc, rec->negb, interior, lo0, hi0, lo1, hi1);
             if (len == 7) s_kernel_tile<7>(planes, rec, lane, acc);
             else if (len == 9) s_kernel_tile<9>(planes, rec, lane, acc);
             else s_kernel_tile<11>(planes, rec, lane, acc);
             int cnt = 0;
             float mn = __int_as_float(0x7f800000);
-            pool_hard(acc, interior, lo0, hi0, lo1, hi1, cnt, mn);
+            pool_hard(acc, cnt, mn);
             publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
             __syncwarp();  // every lane is done with the record before its slot is refilled
             kk = kk_next;
@@ -444,19 +443,15 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                 const TSlotItem si = sh.items[it % kTParamSlots];
                 const KRec* rec = recs + si.rec_slot;
                 const int t0 = si.t0, r0 = si.r0, rg = si.rg, cg = si.cg, box_rows = si.box_rows;
-                const int len = rec->len, d = rec->d, korig = rec->k, lo_u = rec->lo_u, hi_u = rec->hi_u;
+                const int len = rec->len, d = rec->d, korig = rec->k;
                 const int wr = cg == 1 ? warp : (cg == 2 ? warp >> 1 : warp >> 2), wc = warp & (cg - 1);
                 const int lc = kWarpCols * wc + 2 * lane;
                 const bool in_tile = wr < rg;
                 const bool ok0 = in_tile && r0 + lc < d, ok1 = in_tile && r0 + lc + 1 < d;
-                const int u00 = (t0 + kR * wr) * d + r0 + lc, u01 = u00 + 1;
-                const bool mine = ok0 && ok1 && u00 >= lo_u && (u01 + (kR - 1) * d) < hi_u;
-                const bool interior = __all_sync(kFull, mine);
-                int lo0 = 0, hi0 = kR, lo1 = 0, hi1 = kR;
-                if (!interior) {
-                    valid_rows(u00, d, lo_u, hi_u, kR, ok0, lo0, hi0);
-                    valid_rows(u01, d, lo_u, hi_u, kR, ok1, lo1, hi1);
-                }
+                int lo0, hi0, lo1, hi1;
+                valid_rows_tc(t0 + kR * wr, r0 + lc, rec->tl, rec->rl, rec->th, rec->rh, kR, ok0, lo0, hi0);
+                valid_rows_tc(t0 + kR * wr, r0 + lc + 1, rec->tl, rec->rl, rec->th, rec->rh, kR, ok1, lo1, hi1);
+                const bool interior = __all_sync(kFull, lo0 == 0 && lo1 == 0 && hi0 == kR && hi1 == kR);
                 const bool active = __any_sync(kFull, lo0 < hi0 || lo1 < hi1);
                 const int bx = cg == 1 ? 0 : wc >> 1, incol = cg == 1 ? 0 : (wc & 1) * kWarpCols;
                 const int boxw = t_box_cols(cg);
@@ -465,9 +460,7 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                 for (int k = 0; k < 4; ++k)
                     off[k] = t_box_offset(cg, bx, k, box_rows) + 4 * wr * boxw + (((t0 + k) * d) & 3) + incol + 2 * lane;
                 u64 acc[kR];
-                const u64 negb = pack2(rec->negb, rec->negb);
-#pragma unroll
-                for (int o = 0; o < kR; ++o) acc[o] = negb;
+                init_acc(acc, rec->negb, interior, lo0, hi0, lo1, hi1);
                 const bool odd = (d & 1) != 0;
                 if (cg == 1) ok = t_dispatch<kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
                 else ok = t_dispatch<2 * kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
@@ -475,7 +468,7 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                 if (active) {
                     int cnt = 0;
                     float mn = __int_as_float(0x7f800000);
-                    pool_hard(acc, interior, lo0, hi0, lo1, hi1, cnt, mn);
+                    pool_hard(acc, cnt, mn);
                     publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
                 }
                 ++it;

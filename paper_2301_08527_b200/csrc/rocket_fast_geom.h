@@ -25,6 +25,15 @@ ROCKET_HD void valid_rows(int u0, int d, int lo_u, int hi_u, int R, bool col_ok,
     if (!col_ok) o_hi = 0;
 }
 
+// The same without a division, for a column given as (first A-row t_row0, residue c in [0, d)):
+// u = t*d + c >= lo_u = tl*d + rl  <=>  t >= tl + (c < rl), and likewise for the upper end.
+ROCKET_HD void valid_rows_tc(int t_row0, int c, int tl, int rl, int th, int rh, int R, bool col_ok, int& o_lo, int& o_hi) {
+    const int t_lo = tl + (c < rl ? 1 : 0) - t_row0, t_hi = th + (c < rh ? 1 : 0) - t_row0;
+    o_lo = t_lo < 0 ? 0 : (t_lo > R ? R : t_lo);
+    o_hi = t_hi < 0 ? 0 : (t_hi > R ? R : t_hi);
+    if (!col_ok) o_hi = 0;
+}
+
 // S regime: the u of the first output row of raster column cg of a bucket.
 ROCKET_HD int s_column_u0(const SBucket& b, int cg) {
     const int band = cg / b.d, r = cg - band * b.d;

@@ -64,8 +64,11 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
             for (int kk = b.kbeg; kk < b.kend; ++kk) {
                 const KRec& f = plan.krec[kk];
                 REQUIRE(f.d == b.d && kR + f.len - 1 <= b.rows, "S kernel in wrong bucket");
-                int o_lo, o_hi;
-                valid_rows(u0, b.d, f.lo_u, f.hi_u, kR, col_ok, o_lo, o_hi);
+                int o_lo, o_hi, q_lo, q_hi;
+                valid_rows(u0, b.d, f.lo_u, f.hi_u, kR, col_ok, q_lo, q_hi);
+                const int band = cg / b.d;
+                valid_rows_tc(b.tmin + band * kR, cg - band * b.d, f.tl, f.rl, f.th, f.rh, kR, col_ok, o_lo, o_hi);
+                REQUIRE((o_lo >= o_hi && q_lo >= q_hi) || (o_lo == q_lo && o_hi == q_hi), "S row range: the two forms disagree");
                 for (int o = o_lo; o < o_hi; ++o) {
                     const int64_t i = (int64_t)u0 + (int64_t)o * b.d + f.p;
                     REQUIRE(i >= 0 && i < f.nout, "S output out of range");
@@ -118,8 +121,10 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
             const bool col_ok = it.r0 + lc < f.d;
             for (int wr = 0; wr < it.rg; ++wr) {
                 const int u0 = (it.t0 + kR * wr) * f.d + it.r0 + lc;
-                int o_lo, o_hi;
-                valid_rows(u0, f.d, f.lo_u, f.hi_u, kR, col_ok, o_lo, o_hi);
+                int o_lo, o_hi, q_lo, q_hi;
+                valid_rows(u0, f.d, f.lo_u, f.hi_u, kR, col_ok, q_lo, q_hi);
+                valid_rows_tc(it.t0 + kR * wr, it.r0 + lc, f.tl, f.rl, f.th, f.rh, kR, col_ok, o_lo, o_hi);
+                REQUIRE((o_lo >= o_hi && q_lo >= q_hi) || (o_lo == q_lo && o_hi == q_hi), "T row range: the two forms disagree");
                 for (int o = o_lo; o < o_hi; ++o) {
                     const int64_t i = (int64_t)u0 + (int64_t)o * f.d + f.p;
                     REQUIRE(i >= 0 && i < f.nout, "T output out of range");
