@@ -37,6 +37,8 @@ SIGNATURES = {
                                                               ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p,
                                                               ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "rocket_kernel_launch_count": (ctypes.c_int64, []),
+    "rocket_params_set_profiling": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
+    "rocket_params_last_profile": (ctypes.c_int, [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_double)] * 4),
     "rocket_transform": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                         ctypes.c_void_p, ctypes.c_void_p]),
     "rocket_transform_soft": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
@@ -162,6 +164,18 @@ class RocketParams:
         flag = ctypes.c_int()
         _check(load_library().rocket_params_device_status(self._h, flag), "rocket_params_device_status")
         return flag.value
+
+    def set_profiling(self, enable):
+        """rocket_params_set_profiling: record events around the two fused kernels of the hard transform."""
+        _check(load_library().rocket_params_set_profiling(self._h, int(bool(enable))), "rocket_params_set_profiling")
+
+    def last_profile(self):
+        """rocket_params_last_profile: dict with the last call's kernel times (ms) and the per-example
+        conv flop of the two kernels."""
+        v = [ctypes.c_double() for _ in range(4)]
+        _check(load_library().rocket_params_last_profile(self._h, *v), "rocket_params_last_profile")
+        return {"ms_small_dilations": v[0].value, "ms_large_dilations": v[1].value,
+                "flops_small_dilations": v[2].value, "flops_large_dilations": v[3].value}
 
     def set_path(self, path):
         _check(load_library().rocket_params_set_path(self._h, int(path)), "rocket_params_set_path")

@@ -277,6 +277,33 @@ int rocket_params_set_path(rocket_params_t* p, int path) {
     return ROCKET_OK;
 }
 
+int rocket_params_set_profiling(rocket_params_t* p, int enable) {
+    if (!p || enable < 0 || enable > 1) return ROCKET_EINVAL;
+    p->fast->profile = enable != 0;
+    if (!enable) p->fast->ev_valid = false;
+    return ROCKET_OK;
+}
+
+int rocket_params_last_profile(const rocket_params_t* p, double* ms_small_dilations, double* ms_large_dilations,
+                               double* flops_small_dilations, double* flops_large_dilations) {
+    if (!p) return ROCKET_EINVAL;
+    if (flops_small_dilations) *flops_small_dilations = p->fast->host.flops_s;
+    if (flops_large_dilations) *flops_large_dilations = p->fast->host.flops_t;
+    if (ms_small_dilations) *ms_small_dilations = 0.0;
+    if (ms_large_dilations) *ms_large_dilations = 0.0;
+    if (!p->fast->ev_valid || p->device < 0) return ROCKET_OK;
+    DeviceGuard g(p->device);
+    if (!g.ok) return ROCKET_ECUDA;
+    cudaError_t e = cudaEventSynchronize(p->fast->ev[2]);
+    if (e != cudaSuccess) return cuda_status(e);
+    float a = 0.0f, b = 0.0f;
+    if ((e = cudaEventElapsedTime(&a, p->fast->ev[0], p->fast->ev[1])) != cudaSuccess) return cuda_status(e);
+    if ((e = cudaEventElapsedTime(&b, p->fast->ev[1], p->fast->ev[2])) != cudaSuccess) return cuda_status(e);
+    if (ms_small_dilations) *ms_small_dilations = a;
+    if (ms_large_dilations) *ms_large_dilations = b;
+    return ROCKET_OK;
+}
+
 int64_t rocket_kernel_launch_count(void) { return g_launch_count.load(std::memory_order_relaxed); }
 
 int rocket_transform(const rocket_params_t* p, const float* X_dev, int N, int C, int L, float* feat_dev,

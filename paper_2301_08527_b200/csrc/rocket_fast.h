@@ -119,6 +119,7 @@ struct PlanHost {
     std::vector<TMapSpec> tmaps;          // tensor maps the T tiles refer to
     std::vector<int32_t> generic_list;    // kernels the fast path does not take
     int64_t pad_pitch = 0;                // floats per channel row of the zero-margined copy
+    double flops_s = 0.0, flops_t = 0.0;  // conv flop of one example in either regime
 };
 
 struct PlanDevice {
@@ -147,6 +148,9 @@ struct FastState {
     void* maps_blob = nullptr;            // tensor maps
     float* xpad = nullptr;                // padded copy, capacity pad_examples
     int pad_examples = 0;
+    bool profile = false;                 // record events around the S and T launches
+    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+    bool ev_valid = false;
 };
 
 // Uploads the plan (once per handle, at binding).

@@ -592,6 +592,11 @@ void release_fast_state(FastState& fs) {
     if (fs.plan_blob) cudaFree(fs.plan_blob);
     if (fs.maps_blob) cudaFree(fs.maps_blob);
     if (fs.xpad) cudaFree(fs.xpad);
+    for (auto& ev : fs.ev) {
+        if (ev) cudaEventDestroy(ev);
+        ev = nullptr;
+    }
+    fs.ev_valid = false;
     fs.plan_blob = fs.maps_blob = nullptr;
     fs.xpad = nullptr;
     fs.pad_examples = 0;
@@ -672,15 +677,25 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
                                                           fs.host.pad_pitch / 4, kTPadFront / 4);
         count_launch();
     }
+    if (fs.profile) {
+        for (auto& ev : fs.ev)
+            if (!ev && (e = cudaEventCreate(&ev)) != cudaSuccess) return e;
+        cudaEventRecord(fs.ev[0], stream);
+    }
     if (pd.n_sitems > 0) {
         const unsigned long long total = (unsigned long long)N * pd.n_sitems;
         const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms);
         fast_s_forward<<<grid, kSThreads, s_bytes, stream>>>(a);
         count_launch();
     }
+    if (fs.profile) cudaEventRecord(fs.ev[1], stream);
     if (pd.n_titems > 0) {
         fast_t_forward<<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
         count_launch();
+    }
+    if (fs.profile) {
+        cudaEventRecord(fs.ev[2], stream);
+        fs.ev_valid = true;
     }
     const int64_t fin = (int64_t)N * pd.n_krec;
     if (fin > 0) {

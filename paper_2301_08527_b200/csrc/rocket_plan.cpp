@@ -17,6 +17,7 @@ inline int64_t floor_div(int64_t a, int64_t b) { return (a >= 0) ? a / b : -((-a
 
 void build_plan(const HostParams& hp, int split, PlanHost& out) {
     out = PlanHost();
+    out.flops_s = out.flops_t = 0.0;
     if (split < kTMinDilation) split = kTMinDilation;
     out.split = split;
     const int K = hp.K;
@@ -70,6 +71,7 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         for (int k : ks) {
             add_kernel(k);
             const KRec& f = out.krec.back();
+            out.flops_s += 2.0 * f.len * f.m * (double)f.nout;
             tmin = std::min(tmin, floor_div(f.lo_u, d));
             tmax = std::max(tmax, floor_div((int64_t)f.hi_u - 1, d));
             maxlen = std::max(maxlen, f.len);
@@ -103,6 +105,7 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         const int ki = (int)out.krec.size();
         add_kernel(k);
         const KRec f = out.krec.back();
+        out.flops_t += 2.0 * f.len * f.m * (double)f.nout;
         d_max = std::max(d_max, f.d);
         int64_t tmin = floor_div(f.lo_u, f.d);
         const int64_t tmax = floor_div((int64_t)f.hi_u - 1, f.d);
