@@ -35,7 +35,7 @@ LAMBDA, SHIFT = 10.0, 3.0
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the committed ncu capture
 # (profiles/); None until a capture of the current kernel exists.
-NCU_DRAM_BYTES_PER_LAUNCH = {}
+NCU_DRAM_BYTES_PER_LAUNCH = {"fast_s_forward": 38.3e6 * 60 / 8, "fast_t_forward": 64.1e6 * 60 / 8}
 
 
 def fp32_peak_tflops(sm_count, sm_mhz):
