@@ -338,6 +338,14 @@ int rocket_transform_soft(const rocket_params_t* p, const float* X_dev, int N, i
     DeviceGuard g(p->device);
     if (!g.ok) return ROCKET_ECUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const bool aligned = (reinterpret_cast<uintptr_t>(X_dev) & 15u) == 0;
+    if (p->path == 0 && p->fast->host.enabled && aligned) {
+        cudaError_t e = fast::launch_fast_forward(*p->fast, p->dp, X_dev, N, feat_dev, stream, true, lambda, shift, argmax_dev);
+        if (e != cudaSuccess) return cuda_status(e);
+        if (p->fast->dev.n_generic == 0) return ROCKET_OK;
+        return cuda_status(launch_generic_forward(p->dp, X_dev, N, true, lambda, shift, feat_dev, argmax_dev, stream,
+                                                  p->fast->dev.generic_list, p->fast->dev.n_generic));
+    }
     return cuda_status(launch_generic_forward(p->dp, X_dev, N, true, lambda, shift, feat_dev, argmax_dev, stream));
 }
 

@@ -148,6 +148,8 @@ struct FastState {
     void* maps_blob = nullptr;            // tensor maps
     float* xpad = nullptr;                // padded copy, capacity pad_examples
     int pad_examples = 0;
+    void* soft_ws = nullptr;              // soft mode: 16 bytes per (example, kernel), grows with N
+    size_t soft_ws_bytes = 0;
     bool profile = false;                 // record events around the S and T launches
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
     bool ev_valid = false;
@@ -160,9 +162,11 @@ void release_fast_state(FastState& fs);
 // Makes the padded copy hold N examples and (re-)encodes the tensor maps over it.
 cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L);
 
-// Hard forward through the fast path: pad copy, init, S kernel, T kernel, finalise.
+// Forward through the fast path: init, pad copy, S kernel, T kernel, finalise.  soft = false:
+// PPV + max; soft = true: softPPV + max (+ argmax when argmax != nullptr).
 cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const float* X, int N, float* feat,
-                                cudaStream_t stream);
+                                cudaStream_t stream, bool soft = false, float lambda = 0.0f, float shift = 0.0f,
+                                int32_t* argmax = nullptr);
 
 }  // namespace fast
 }  // namespace rocket

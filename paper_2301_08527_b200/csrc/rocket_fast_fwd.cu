@@ -1,4 +1,5 @@
-// Fused forward kernels of the fast path (hard PPV + max): see rocket_fast.h for the geometry.
+// Fused forward kernels of the fast path (hard PPV + max, soft PPV + max + argmax): see rocket_fast.h
+// for the geometry.
 //
 // Arithmetic conventions shared by both kernels
 //   - Accumulators hold -z: weights and bias are stored negated (acc = (0 - b) + sum (-w) x).  Then
@@ -122,12 +123,87 @@ __device__ __forceinline__ void publish(int* __restrict__ feat_i, int64_t pair, 
     }
 }
 
+__device__ __forceinline__ u64 add2(u64 a, u64 b) {
+    u64 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ float ex2_approx(float v) {
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
+}
+__device__ __forceinline__ float rcp_approx(float v) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
+}
+
+constexpr float kSoftFixedScale = 1073741824.0f;  // 2^30: soft sums travel as fixed-point integers
+
+// Soft pooling of a warp tile (Eq. 3-4): sum of h = 1 / (1 + 2^(c1 * acc + c0)) over the valid
+// outputs (acc = -z, c1 = lambda * log2 e, c0 = -shift * log2 e), the max and the lowest output
+// index attaining it.  base0 / base1 are the output indices of row 0 of the thread's two columns,
+// step the index distance between rows.  The warp's sum is added to ws[2 * pair] as a fixed-point
+// integer and (max key, INT_MAX - index) is folded into ws[2 * pair + 1] with one 64-bit atomic max:
+// both are exact and order-free, so results are run-to-run identical.
+__device__ __forceinline__ void pool_publish_soft(unsigned long long* __restrict__ ws, int64_t pair, const u64 (&acc)[kR],
+                                                  float c1, float c0, bool interior, int lo0, int hi0, int lo1, int hi1,
+                                                  int base0, int base1, int step, int lane) {
+    const u64 c1p = pack2(c1, c1), c0p = pack2(c0, c0), one = pack2(1.0f, 1.0f);
+    u64 hs = pack2(0.0f, 0.0f);
+    float mn = __int_as_float(0x7f800000);
+#pragma unroll
+    for (int o = 0; o < kR; ++o) {
+        u64 t = c0p;
+        fma2(t, acc[o], c1p);
+        float ta, tb, a, b;
+        unpack2(t, ta, tb);
+        const u64 den = add2(pack2(ex2_approx(ta), ex2_approx(tb)), one);
+        unpack2(den, ta, tb);
+        float ha = rcp_approx(ta), hb = rcp_approx(tb);
+        if (!interior) {
+            if (o < lo0 || o >= hi0) ha = 0.0f;
+            if (o < lo1 || o >= hi1) hb = 0.0f;
+        }
+        hs = add2(hs, pack2(ha, hb));
+        unpack2(acc[o], a, b);
+        mn = min3(mn, a, b);
+    }
+    float h0, h1;
+    unpack2(hs, h0, h1);
+    float hsum = h0 + h1;
+#pragma unroll
+    for (int sh = 16; sh > 0; sh >>= 1) hsum += __shfl_xor_sync(kFull, hsum, sh);
+    const int key = float_key(-mn);
+    const int wkey = __reduce_max_sync(kFull, key);
+    int idx = INT_MAX;
+    if (key == wkey) {
+#pragma unroll
+        for (int o = kR - 1; o >= 0; --o) {
+            float a, b;
+            unpack2(acc[o], a, b);
+            if (b == mn) idx = min(idx, base1 + o * step);
+            if (a == mn) idx = min(idx, base0 + o * step);
+        }
+    }
+    idx = __reduce_min_sync(kFull, idx);
+    if (lane == 0) {
+        atomicAdd(ws + 2 * pair, __float2ull_rn(hsum * kSoftFixedScale));
+        const unsigned long long k64 = ((unsigned long long)((unsigned)wkey ^ 0x80000000u) << 32) |
+                                       (unsigned long long)(unsigned)(INT_MAX - idx);
+        atomicMax(ws + 2 * pair + 1, k64);
+    }
+}
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 struct FwdArgs {
     PlanDevice plan;
     const float* X;
     int* feat_i;
+    unsigned long long* ws;  // soft mode: (fixed-point sum, max key and index) per (example, kernel)
+    float c1, c0;            // soft mode: lambda * log2 e, -shift * log2 e
     int N, C, L, K;
 };
 
@@ -152,6 +228,7 @@ __device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* r
         conv_channel<ELL, false, 4 * kWarpCols>(planes + rec->ch[q] * kSPlaneFloats, off, rec->w2[q], acc);
 }
 
+template <bool SOFT>
 __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
     float* planes = reinterpret_cast<float*>(smem_raw);                               // [C][kRowsMax][64]
     KRec* recs = reinterpret_cast<KRec*>(planes + a.C * kSPlaneFloats);                // [warps][2]
@@ -237,10 +314,16 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
             if (len == 7) s_kernel_tile<7>(planes, rec, lane, acc);
             else if (len == 9) s_kernel_tile<9>(planes, rec, lane, acc);
             else s_kernel_tile<11>(planes, rec, lane, acc);
-            int cnt = 0;
-            float mn = __int_as_float(0x7f800000);
-            pool_hard(acc, cnt, mn);
-            publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
+            if (SOFT) {
+                const int p = rec->p;
+                pool_publish_soft(a.ws, (int64_t)n * a.K + korig, acc, a.c1, a.c0, interior, lo0, hi0, lo1, hi1,
+                                  trow0 * d + c0 + p, trow1 * d + c1 + p, d, lane);
+            } else {
+                int cnt = 0;
+                float mn = __int_as_float(0x7f800000);
+                pool_hard(acc, cnt, mn);
+                publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
+            }
             __syncwarp();  // every lane is done with the record before its slot is refilled
             kk = kk_next;
             cur ^= 1;
@@ -336,6 +419,7 @@ __device__ __forceinline__ bool t_dispatch(int len, bool odd, const float* stage
                : t_channels<11, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
 }
 
+template <bool SOFT>
 __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
     __shared__ __align__(16) TShared sh;
     // dynamic shared memory, aligned to 128 bytes by hand: stages, then kernel-record slots
@@ -466,10 +550,16 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                 else ok = t_dispatch<2 * kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
                 if (!ok) break;
                 if (active) {
-                    int cnt = 0;
-                    float mn = __int_as_float(0x7f800000);
-                    pool_hard(acc, cnt, mn);
-                    publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
+                    if (SOFT) {
+                        const int base = (t0 + kR * wr) * d + r0 + lc + rec->p;
+                        pool_publish_soft(a.ws, (int64_t)n * a.K + korig, acc, a.c1, a.c0, interior, lo0, hi0, lo1, hi1, base,
+                                          base + 1, d, lane);
+                    } else {
+                        int cnt = 0;
+                        float mn = __int_as_float(0x7f800000);
+                        pool_hard(acc, cnt, mn);
+                        publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
+                    }
                 }
                 ++it;
             }
@@ -511,6 +601,26 @@ __global__ void fast_finalize_kernel(float* __restrict__ feat, const KRec* __res
     const int cnt = fi[0], key = fi[1];
     feat[((int64_t)n * K + k) * 2] = (float)cnt / (float)nout;   // Eq. 2
     feat[((int64_t)n * K + k) * 2 + 1] = key_float(key);
+}
+
+__global__ void fast_init_soft_kernel(unsigned long long* __restrict__ ws, int64_t pairs, unsigned* counters) {
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e == 0) { counters[0] = 0u; counters[1] = 0u; }
+    if (e < pairs) { ws[2 * e] = 0ull; ws[2 * e + 1] = 0ull; }
+}
+
+__global__ void fast_finalize_soft_kernel(float* __restrict__ feat, int32_t* __restrict__ argmax,
+                                          const unsigned long long* __restrict__ ws, const KRec* __restrict__ krec,
+                                          int n_krec, int N, int K) {
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= (int64_t)N * n_krec) return;
+    const int n = (int)(e / n_krec), f = (int)(e - (int64_t)n * n_krec);
+    const int k = krec[f].k, nout = krec[f].nout;
+    const int64_t pair = (int64_t)n * K + k;
+    const unsigned long long sum = ws[2 * pair], k64 = ws[2 * pair + 1];
+    feat[pair * 2] = (float)((double)sum / (double)kSoftFixedScale / (double)nout);   // Eq. 4
+    feat[pair * 2 + 1] = key_float((int)((unsigned)(k64 >> 32) ^ 0x80000000u));
+    if (argmax) argmax[pair] = INT_MAX - (int)(unsigned)(k64 & 0xffffffffull);
 }
 
 size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
@@ -592,6 +702,9 @@ void release_fast_state(FastState& fs) {
     if (fs.plan_blob) cudaFree(fs.plan_blob);
     if (fs.maps_blob) cudaFree(fs.maps_blob);
     if (fs.xpad) cudaFree(fs.xpad);
+    if (fs.soft_ws) cudaFree(fs.soft_ws);
+    fs.soft_ws = nullptr;
+    fs.soft_ws_bytes = 0;
     for (auto& ev : fs.ev) {
         if (ev) cudaEventDestroy(ev);
         ev = nullptr;
@@ -643,7 +756,7 @@ cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L) {
 }
 
 cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const float* X, int N, float* feat,
-                                cudaStream_t stream) {
+                                cudaStream_t stream, bool soft, float lambda, float shift, int32_t* argmax) {
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -653,9 +766,13 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
     bool& attr_done = attr_done_for[dev & 63];
     const size_t s_bytes = s_smem_bytes(dp.C), t_bytes = t_smem_bytes();
     if (!attr_done) {
-        e = cudaFuncSetAttribute(fast_s_forward, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s_smem_bytes(kSMaxChannels));
+        e = cudaFuncSetAttribute(fast_s_forward<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s_smem_bytes(kSMaxChannels));
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(fast_t_forward, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t_bytes);
+        e = cudaFuncSetAttribute(fast_s_forward<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s_smem_bytes(kSMaxChannels));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(fast_t_forward<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t_bytes);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(fast_t_forward<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t_bytes);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -664,11 +781,22 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
         e = ensure_pad_capacity(fs, N, dp.C, dp.L);
         if (e != cudaSuccess) return e;
     }
+    const int64_t pairs = (int64_t)N * dp.K;
+    if (soft && (size_t)pairs * 16 > fs.soft_ws_bytes) {
+        if (fs.soft_ws) cudaFree(fs.soft_ws);  // waits for work that still uses it
+        fs.soft_ws = nullptr;
+        fs.soft_ws_bytes = 0;
+        e = cudaMalloc(&fs.soft_ws, (size_t)pairs * 16);
+        if (e != cudaSuccess) { fs.soft_ws = nullptr; return e; }
+        fs.soft_ws_bytes = (size_t)pairs * 16;
+    }
     FwdArgs a;
     a.plan = fs.dev; a.X = X; a.feat_i = reinterpret_cast<int*>(feat);
+    a.ws = static_cast<unsigned long long*>(fs.soft_ws);
+    a.c1 = lambda * 1.4426950408889634f; a.c0 = -shift * 1.4426950408889634f;
     a.N = N; a.C = dp.C; a.L = dp.L; a.K = dp.K;
-    const int64_t pairs = (int64_t)N * dp.K;
-    fast_init_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, stream>>>(a.feat_i, pairs, pd.counters);
+    if (soft) fast_init_soft_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, stream>>>(a.ws, pairs, pd.counters);
+    else fast_init_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, stream>>>(a.feat_i, pairs, pd.counters);
     count_launch();
     if (pd.n_titems > 0) {
         const int64_t rows = (int64_t)N * dp.C;
@@ -685,12 +813,14 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
     if (pd.n_sitems > 0) {
         const unsigned long long total = (unsigned long long)N * pd.n_sitems;
         const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms);
-        fast_s_forward<<<grid, kSThreads, s_bytes, stream>>>(a);
+        if (soft) fast_s_forward<true><<<grid, kSThreads, s_bytes, stream>>>(a);
+        else fast_s_forward<false><<<grid, kSThreads, s_bytes, stream>>>(a);
         count_launch();
     }
     if (fs.profile) cudaEventRecord(fs.ev[1], stream);
     if (pd.n_titems > 0) {
-        fast_t_forward<<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
+        if (soft) fast_t_forward<true><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
+        else fast_t_forward<false><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
         count_launch();
     }
     if (fs.profile) {
@@ -699,7 +829,8 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
     }
     const int64_t fin = (int64_t)N * pd.n_krec;
     if (fin > 0) {
-        fast_finalize_kernel<<<(unsigned)((fin + 255) / 256), 256, 0, stream>>>(feat, pd.krec, pd.n_krec, N, dp.K);
+        if (soft) fast_finalize_soft_kernel<<<(unsigned)((fin + 255) / 256), 256, 0, stream>>>(feat, argmax, a.ws, pd.krec, pd.n_krec, N, dp.K);
+        else fast_finalize_kernel<<<(unsigned)((fin + 255) / 256), 256, 0, stream>>>(feat, pd.krec, pd.n_krec, N, dp.K);
         count_launch();
     }
     return cudaGetLastError();
