@@ -362,6 +362,10 @@ int rocket_transform_soft_backward(const rocket_params_t* p, const float* X_dev,
     if (!g.ok) return ROCKET_ECUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int64_t nW = n_weights_of(p);
+    const bool aligned = (reinterpret_cast<uintptr_t>(X_dev) & 15u) == 0;
+    if (p->path == 0 && p->fast->host.enabled && p->fast->host.generic_list.empty() && (aligned || N == 0))
+        return cuda_status(fast::launch_fast_backward(*p->fast, p->dp, nW, X_dev, N, lambda, shift, dfeat_dev, argmax_dev,
+                                                      dW_dev, db_dev, stream));
     float* scratch = nullptr;
     if (N > 0) {
         std::lock_guard<std::mutex> lk(p->mu);

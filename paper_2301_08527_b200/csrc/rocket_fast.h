@@ -53,7 +53,8 @@ struct alignas(16) KRec {
     float negb;                    // 0 - bias (never -0.0)
     int32_t ch[ROCKET_MAX_CHANNELS_PER_KERNEL];
     int32_t tl, rl, th, rh;        // lo_u = tl * d + rl and hi_u = th * d + rh with 0 <= rl, rh < d
-    int32_t pad_[8];
+    int32_t woff;                  // offset of the kernel's weights in the caller's ragged weight array
+    int32_t pad_[7];
     // w2[q][2j] = w2[q][2j+1] = 0 - W[q][j]: each weight twice, ready as a packed pair
     float w2[ROCKET_MAX_CHANNELS_PER_KERNEL][kPairRow];
 };
@@ -150,6 +151,7 @@ struct FastState {
     int pad_examples = 0;
     void* soft_ws = nullptr;              // soft mode: 16 bytes per (example, kernel), grows with N
     size_t soft_ws_bytes = 0;
+    void* bwd_ws = nullptr;               // backward: fixed-point sums [n_weights + K], scales [K], max |x|
     bool profile = false;                 // record events around the S and T launches
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
     bool ev_valid = false;
@@ -161,6 +163,12 @@ cudaError_t upload_plan(FastState& fs);
 void release_fast_state(FastState& fs);
 // Makes the padded copy hold N examples and (re-)encodes the tensor maps over it.
 cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L);
+
+// Backward of the soft transform through the fast path (every kernel must be a fast-path kernel):
+// dW (ragged like the weights, n_weights floats) and db [K] are assigned.
+cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t n_weights, const float* X, int N,
+                                 float lambda, float shift, const float* dfeat, const int32_t* argmax, float* dW,
+                                 float* db, cudaStream_t stream);
 
 // Forward through the fast path: init, pad copy, S kernel, T kernel, finalise.  soft = false:
 // PPV + max; soft = true: softPPV + max (+ argmax when argmax != nullptr).

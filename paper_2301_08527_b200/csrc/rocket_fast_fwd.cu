@@ -196,6 +196,105 @@ __device__ __forceinline__ void pool_publish_soft(unsigned long long* __restrict
     }
 }
 
+__device__ __forceinline__ u64 mul2(u64 a, u64 b) {
+    u64 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+// Backward, first half: turns the accumulators (acc = -z) of a warp tile into
+//   gz = gPs * h (1 - h) + gM [output index == argmax],  h = 1 / (1 + 2^(c1 * acc + c0)),
+// zero where the output does not exist, and returns the thread's sum of gz (its share of db).
+// oA0 / oA1: the row of the thread's first / second column that is the argmax, or -1.
+__device__ __forceinline__ float make_gz(u64 (&acc)[kR], float c1, float c0, float gPs, float gM, bool interior, int lo0,
+                                         int hi0, int lo1, int hi1, int oA0, int oA1) {
+    const u64 c1p = pack2(c1, c1), c0p = pack2(c0, c0), one = pack2(1.0f, 1.0f), neg1 = pack2(-1.0f, -1.0f);
+    const u64 gp = pack2(gPs, gPs);
+    u64 sum = pack2(0.0f, 0.0f);
+#pragma unroll
+    for (int o = 0; o < kR; ++o) {
+        u64 t = c0p;
+        fma2(t, acc[o], c1p);
+        float ta, tb;
+        unpack2(t, ta, tb);
+        const u64 den = add2(pack2(ex2_approx(ta), ex2_approx(tb)), one);
+        unpack2(den, ta, tb);
+        const u64 hh = pack2(rcp_approx(ta), rcp_approx(tb));
+        u64 omh = one;
+        fma2(omh, hh, neg1);                      // 1 - h
+        u64 g = mul2(mul2(hh, omh), gp);
+        float ga, gb;
+        unpack2(g, ga, gb);
+        if (!interior) {
+            if (o < lo0 || o >= hi0) ga = 0.0f;
+            if (o < lo1 || o >= hi1) gb = 0.0f;
+        }
+        if (o == oA0) ga += gM;
+        if (o == oA1) gb += gM;
+        g = pack2(ga, gb);
+        acc[o] = g;
+        sum = add2(sum, g);
+    }
+    float s0, s1;
+    unpack2(sum, s0, s1);
+    return s0 + s1;
+}
+
+// Backward, second half, one channel of one warp tile: dw[j] += gz[o] * x[o + j] for the thread's
+// column pair (same traversal as conv_channel with the roles of weights and accumulators swapped).
+template <int ELL, bool ODD, int STEP>
+__device__ __forceinline__ void grad_channel(const float* __restrict__ st, const int (&off)[4], const u64 (&gz)[kR],
+                                             u64 (&dw)[ELL]) {
+#pragma unroll
+    for (int s = 0; s < kR + ELL - 1; ++s) {
+        const float* p = st + off[s & 3] + (s >> 2) * STEP;
+        u64 x;
+        if (ODD && (s & 1)) x = pack2(p[0], p[1]);
+        else x = *reinterpret_cast<const u64*>(p);
+#pragma unroll
+        for (int j = 0; j < ELL; ++j) {
+            const int o = s - j;
+            if (o >= 0 && o < kR) fma2(dw[j], gz[o], x);
+        }
+    }
+}
+
+// Adds a float to a fixed-point accumulator (value * scale as a 64-bit integer): exact and order-free.
+__device__ __forceinline__ void add_fixed(long long* dst, float v, double scale) {
+    atomicAdd(reinterpret_cast<unsigned long long*>(dst), (unsigned long long)__double2ll_rn((double)v * scale));
+}
+
+// Sums dw[j] (both halves) over the warp and adds the ELL totals to dst[0..ELL).  A butterfly that
+// halves the number of live values at every step leaves total j on the lanes with (lane >> 1) == j.
+template <int ELL>
+__device__ __forceinline__ void reduce_publish_dw(const u64 (&dw)[ELL], long long* dst, double scale, int lane) {
+    float v[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        if (j < ELL) {
+            float a, b;
+            unpack2(dw[j], a, b);
+            v[j] = a + b;
+        } else {
+            v[j] = 0.0f;
+        }
+    }
+#pragma unroll
+    for (int half = 8; half >= 1; half >>= 1) {
+        const int mask = half * 2;
+        const bool up = (lane & mask) != 0;
+#pragma unroll
+        for (int i = 0; i < half; ++i) {
+            const float send = up ? v[i] : v[i + half];
+            const float keep = up ? v[i + half] : v[i];
+            v[i] = keep + __shfl_xor_sync(kFull, send, mask);
+        }
+    }
+    const float total = v[0] + __shfl_xor_sync(kFull, v[0], 1);
+    const int j = lane >> 1;
+    if ((lane & 1) == 0 && j < ELL) add_fixed(dst + j, total, scale);
+}
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 struct FwdArgs {
@@ -205,6 +304,13 @@ struct FwdArgs {
     unsigned long long* ws;  // soft mode: (fixed-point sum, max key and index) per (example, kernel)
     float c1, c0;            // soft mode: lambda * log2 e, -shift * log2 e
     int N, C, L, K;
+    // backward
+    const float* dfeat;      // [N][2K]
+    const int32_t* argmax;   // [N][K]
+    long long* accfix;       // fixed-point sums: dW ragged [n_weights], then db [K]
+    const double* scale;     // [K] fixed-point scale of every kernel's sums
+    long long n_weights;
+    float lambda;
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -220,6 +326,21 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+// Backward second half for one kernel on an S tile: per channel, dW sums of the warp tile.
+template <int ELL>
+__device__ __forceinline__ void s_grad_tile(const float* planes, const KRec* rec, int lane, const u64 (&gz)[kR],
+                                            long long* accfix, double scale) {
+    const int m = rec->m;
+    const int off[4] = {2 * lane, kWarpCols + 2 * lane, 2 * kWarpCols + 2 * lane, 3 * kWarpCols + 2 * lane};
+    for (int q = 0; q < m; ++q) {
+        u64 dw[ELL];
+#pragma unroll
+        for (int j = 0; j < ELL; ++j) dw[j] = 0ull;
+        grad_channel<ELL, false, 4 * kWarpCols>(planes + rec->ch[q] * kSPlaneFloats, off, gz, dw);
+        reduce_publish_dw<ELL>(dw, accfix + rec->woff + q * ELL, scale, lane);
+    }
+}
+
 template <int ELL>
 __device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* rec, int lane, u64 (&acc)[kR]) {
     const int m = rec->m;
@@ -228,7 +349,7 @@ __device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* r
         conv_channel<ELL, false, 4 * kWarpCols>(planes + rec->ch[q] * kSPlaneFloats, off, rec->w2[q], acc);
 }
 
-template <bool SOFT>
+template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft
 __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
     float* planes = reinterpret_cast<float*>(smem_raw);                               // [C][kRowsMax][64]
     KRec* recs = reinterpret_cast<KRec*>(planes + a.C * kSPlaneFloats);                // [warps][2]
@@ -314,7 +435,22 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
             if (len == 7) s_kernel_tile<7>(planes, rec, lane, acc);
             else if (len == 9) s_kernel_tile<9>(planes, rec, lane, acc);
             else s_kernel_tile<11>(planes, rec, lane, acc);
-            if (SOFT) {
+            if (MODE == 2) {
+                const int64_t pair = (int64_t)n * a.K + korig;
+                const float gP = __ldg(a.dfeat + 2 * pair), gM = __ldg(a.dfeat + 2 * pair + 1);
+                const int uA = __ldg(a.argmax + pair) - rec->p;
+                const int tA = (uA + 8 * d) / d - 8, cA = uA - tA * d;   // uA >= -p > -8 d
+                const int oA0 = (ok0 && c0 == cA && tA >= trow0 && tA < trow0 + kR) ? tA - trow0 : -1;
+                const int oA1 = (ok1 && c1 == cA && tA >= trow1 && tA < trow1 + kR) ? tA - trow1 : -1;
+                float dbs = make_gz(acc, a.c1, a.c0, gP * a.lambda / (float)rec->nout, gM, interior, lo0, hi0, lo1, hi1, oA0, oA1);
+#pragma unroll
+                for (int sh = 16; sh > 0; sh >>= 1) dbs += __shfl_xor_sync(kFull, dbs, sh);
+                const double scale = __ldg(a.scale + korig);
+                if (lane == 0) add_fixed(a.accfix + a.n_weights + korig, dbs, scale);
+                if (len == 7) s_grad_tile<7>(planes, rec, lane, acc, a.accfix, scale);
+                else if (len == 9) s_grad_tile<9>(planes, rec, lane, acc, a.accfix, scale);
+                else s_grad_tile<11>(planes, rec, lane, acc, a.accfix, scale);
+            } else if (MODE == 1) {
                 const int p = rec->p;
                 pool_publish_soft(a.ws, (int64_t)n * a.K + korig, acc, a.c1, a.c0, interior, lo0, hi0, lo1, hi1,
                                   trow0 * d + c0 + p, trow1 * d + c1 + p, d, lane);
@@ -407,6 +543,44 @@ __device__ __forceinline__ bool t_channels(const float* stages, const KRec* rec,
     return true;
 }
 
+// Backward second half on a T tile: the kernel's channels stream through the ring once more.
+template <int ELL, bool ODD, int STEP>
+__device__ __forceinline__ bool t_grad_channels(const float* stages, const KRec* rec, const int (&off)[4], uint32_t full0,
+                                                uint32_t empty0, uint32_t& st, int lane, bool active, const u64 (&gz)[kR],
+                                                long long* accfix, double scale) {
+    const int m = rec->m;
+    for (int q = 0; q < m; ++q) {
+        const uint32_t slot = st % kTStages;
+        if (!mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) return false;
+        if (active) {
+            u64 dw[ELL];
+#pragma unroll
+            for (int j = 0; j < ELL; ++j) dw[j] = 0ull;
+            grad_channel<ELL, ODD, STEP>(stages + slot * kTStageFloats, off, gz, dw);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8u * slot);
+            reduce_publish_dw<ELL>(dw, accfix + rec->woff + q * ELL, scale, lane);
+        } else {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8u * slot);
+        }
+        ++st;
+    }
+    return true;
+}
+
+template <int STEP>
+__device__ __forceinline__ bool t_grad_dispatch(int len, bool odd, const float* stages, const KRec* rec, const int (&off)[4],
+                                                uint32_t full0, uint32_t empty0, uint32_t& st, int lane, bool active,
+                                                const u64 (&gz)[kR], long long* accfix, double scale) {
+    if (len == 7) return odd ? t_grad_channels<7, true, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale)
+                             : t_grad_channels<7, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale);
+    if (len == 9) return odd ? t_grad_channels<9, true, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale)
+                             : t_grad_channels<9, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale);
+    return odd ? t_grad_channels<11, true, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale)
+               : t_grad_channels<11, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale);
+}
+
 template <int STEP>
 __device__ __forceinline__ bool t_dispatch(int len, bool odd, const float* stages, const KRec* rec, const int (&off)[4],
                                            uint32_t full0, uint32_t empty0, uint32_t& st, int lane, bool active,
@@ -419,7 +593,7 @@ __device__ __forceinline__ bool t_dispatch(int len, bool odd, const float* stage
                : t_channels<11, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
 }
 
-template <bool SOFT>
+template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft
 __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
     __shared__ __align__(16) TShared sh;
     // dynamic shared memory, aligned to 128 bytes by hand: stages, then kernel-record slots
@@ -473,7 +647,9 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                     const bool new_rec = krec != cur_krec;
                     if (new_rec) { cur_krec = krec; ++nrec; }
                     const uint32_t rslot = (nrec - 1u) % kTParamSlots;
-                    for (int q = 0; q < m; ++q) {
+                    const int n_stages = MODE == 2 ? 2 * m : m;   // the backward streams the channels twice
+                    for (int q2 = 0; q2 < n_stages; ++q2) {
+                        const int q = q2 < m ? q2 : q2 - m;
                         const uint32_t slot = st % kTStages;
                         if (st >= (uint32_t)kTStages && !mbar_wait(empty0 + 8u * slot, ((st / kTStages) - 1u) & 1u)) {
                             ok = false;
@@ -481,13 +657,13 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                         }
                         const uint32_t bar = full0 + 8u * slot;
                         uint32_t tx = (uint32_t)nbx * 4u * box_bytes;
-                        if (q == 0) {
+                        if (q2 == 0) {
                             TSlotItem& si = sh.items[it % kTParamSlots];
                             si.t0 = t0; si.r0 = r0; si.rg = rg; si.cg = cg; si.box_rows = box_rows; si.rec_slot = (int)rslot;
                             if (new_rec) tx += (uint32_t)sizeof(KRec);
                         }
                         mbar_arrive_expect_tx(bar, tx);
-                        if (q == 0 && new_rec) bulk_g2s(smem_u32(recs + rslot), a.plan.krec + krec, (uint32_t)sizeof(KRec), bar);
+                        if (q2 == 0 && new_rec) bulk_g2s(smem_u32(recs + rslot), a.plan.krec + krec, (uint32_t)sizeof(KRec), bar);
                         const int ch = (int)((chw[q >> 2] >> (8 * (q & 3))) & 0xffu);
                         const int z = n * a.C + ch;
                         const uint32_t dst0 = smem_u32(stages + slot * kTStageFloats);
@@ -549,8 +725,31 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                 if (cg == 1) ok = t_dispatch<kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
                 else ok = t_dispatch<2 * kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
                 if (!ok) break;
-                if (active) {
-                    if (SOFT) {
+                if (MODE == 2) {
+                    const int64_t pair = (int64_t)n * a.K + korig;
+                    double scale = 0.0;
+                    if (active) {
+                        const float gP = __ldg(a.dfeat + 2 * pair), gM = __ldg(a.dfeat + 2 * pair + 1);
+                        const int uA = __ldg(a.argmax + pair) - rec->p;
+                        const int tA = (uA + 8 * d) / d - 8, cA = uA - tA * d;   // uA >= -p > -8 d
+                        const int trow = t0 + kR * wr, c0 = r0 + lc;
+                        const bool rowhit = tA >= trow && tA < trow + kR;
+                        const int oA0 = (ok0 && rowhit && c0 == cA) ? tA - trow : -1;
+                        const int oA1 = (ok1 && rowhit && c0 + 1 == cA) ? tA - trow : -1;
+                        float dbs = make_gz(acc, a.c1, a.c0, gP * a.lambda / (float)rec->nout, gM, interior, lo0, hi0, lo1, hi1, oA0,
+                                            oA1);
+#pragma unroll
+                        for (int sh = 16; sh > 0; sh >>= 1) dbs += __shfl_xor_sync(kFull, dbs, sh);
+                        scale = __ldg(a.scale + korig);
+                        if (lane == 0) add_fixed(a.accfix + a.n_weights + korig, dbs, scale);
+                    }
+                    if (cg == 1) ok = t_grad_dispatch<kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc,
+                                                                     a.accfix, scale);
+                    else ok = t_grad_dispatch<2 * kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc,
+                                                                 a.accfix, scale);
+                    if (!ok) break;
+                } else if (active) {
+                    if (MODE == 1) {
                         const int base = (t0 + kR * wr) * d + r0 + lc + rec->p;
                         pool_publish_soft(a.ws, (int64_t)n * a.K + korig, acc, a.c1, a.c0, interior, lo0, hi0, lo1, hi1, base,
                                           base + 1, d, lane);
@@ -644,6 +843,76 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
+// Opts every fused kernel into its dynamic shared memory size, once per device.
+cudaError_t set_kernel_attributes(int dev) {
+    cudaError_t e = cudaSuccess;
+    static bool attr_done_for[64] = {};
+    bool& attr_done = attr_done_for[dev & 63];
+    const size_t t_bytes = t_smem_bytes();
+    if (!attr_done) {
+        e = cudaFuncSetAttribute(fast_s_forward<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s_smem_bytes(kSMaxChannels));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(fast_s_forward<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s_smem_bytes(kSMaxChannels));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(fast_t_forward<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t_bytes);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(fast_t_forward<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t_bytes);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(fast_s_forward<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s_smem_bytes(kSMaxChannels));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(fast_t_forward<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t_bytes);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    return cudaSuccess;
+}
+
+// ---- backward helpers ----------------------------------------------------------------------------
+// Largest |x| of the batch, as the bit pattern of a non-negative float (integer order = float order).
+__global__ void fast_absmax_kernel(const float4* __restrict__ X, int64_t n4, unsigned* __restrict__ out) {
+    float m = 0.0f;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n4; e += (int64_t)gridDim.x * blockDim.x) {
+        const float4 v = __ldg(X + e);
+        m = fmaxf(fmaxf(m, fabsf(v.x)), fmaxf(fabsf(v.y), fmaxf(fabsf(v.z), fabsf(v.w))));
+    }
+    unsigned b = __float_as_uint(m);
+    b = __reduce_max_sync(kFull, b);
+    if ((threadIdx.x & 31) == 0) atomicMax(out, b);
+}
+
+// Per kernel: a bound on sum |gz| |x| over the batch gives the fixed-point scale of its sums
+// (|sum_i gz_i| <= |gP| lambda / 4 + |gM| per example since h (1 - h) <= 1/4), and its sums are cleared.
+__global__ void fast_bwd_prepare_kernel(const float* __restrict__ dfeat, const KRec* __restrict__ krec, int n_krec, int N,
+                                        int K, float lambda, const unsigned* __restrict__ absmax_bits,
+                                        double* __restrict__ scale, long long* __restrict__ accfix, long long n_weights) {
+    const int f = blockIdx.x * blockDim.x + threadIdx.x;
+    if (f >= n_krec) return;
+    const int k = krec[f].k;
+    double bound = 0.0;
+    for (int n = 0; n < N; ++n) {
+        const float gP = dfeat[((int64_t)n * K + k) * 2], gM = dfeat[((int64_t)n * K + k) * 2 + 1];
+        bound += (double)fabsf(gP) * (double)fabsf(lambda) * 0.25 + (double)fabsf(gM);
+    }
+    const double xmax = fmax((double)__uint_as_float(*absmax_bits), 1.0);
+    bound *= xmax * 1.01;
+    scale[k] = (bound > 0.0 && bound < 1e300) ? 1152921504606846976.0 / bound : 0.0;  // 2^60 / bound
+    const int taps = krec[f].m * krec[f].len;
+    for (int t = 0; t < taps; ++t) accfix[krec[f].woff + t] = 0;
+    accfix[n_weights + k] = 0;
+}
+
+__global__ void fast_bwd_finalize_kernel(const long long* __restrict__ accfix, const double* __restrict__ scale,
+                                         const KRec* __restrict__ krec, int n_krec, long long n_weights,
+                                         float* __restrict__ dW, float* __restrict__ db) {
+    const int f = blockIdx.x * blockDim.x + threadIdx.x;
+    if (f >= n_krec) return;
+    const int k = krec[f].k;
+    const double sc = scale[k], inv = sc > 0.0 ? 1.0 / sc : 0.0;
+    const int taps = krec[f].m * krec[f].len;
+    for (int t = 0; t < taps; ++t) dW[krec[f].woff + t] = (float)((double)accfix[krec[f].woff + t] * inv);
+    db[k] = (float)((double)accfix[n_weights + k] * inv);
+}
+
 }  // namespace
 
 cudaError_t upload_plan(FastState& fs) {
@@ -703,6 +972,8 @@ void release_fast_state(FastState& fs) {
     if (fs.maps_blob) cudaFree(fs.maps_blob);
     if (fs.xpad) cudaFree(fs.xpad);
     if (fs.soft_ws) cudaFree(fs.soft_ws);
+    if (fs.bwd_ws) cudaFree(fs.bwd_ws);
+    fs.bwd_ws = nullptr;
     fs.soft_ws = nullptr;
     fs.soft_ws_bytes = 0;
     for (auto& ev : fs.ev) {
@@ -762,20 +1033,9 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    static bool attr_done_for[64] = {};
-    bool& attr_done = attr_done_for[dev & 63];
+    e = set_kernel_attributes(dev);
+    if (e != cudaSuccess) return e;
     const size_t s_bytes = s_smem_bytes(dp.C), t_bytes = t_smem_bytes();
-    if (!attr_done) {
-        e = cudaFuncSetAttribute(fast_s_forward<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s_smem_bytes(kSMaxChannels));
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(fast_s_forward<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s_smem_bytes(kSMaxChannels));
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(fast_t_forward<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t_bytes);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(fast_t_forward<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t_bytes);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
     const PlanDevice& pd = fs.dev;
     if (pd.n_titems > 0) {
         e = ensure_pad_capacity(fs, N, dp.C, dp.L);
@@ -795,6 +1055,7 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
     a.ws = static_cast<unsigned long long*>(fs.soft_ws);
     a.c1 = lambda * 1.4426950408889634f; a.c0 = -shift * 1.4426950408889634f;
     a.N = N; a.C = dp.C; a.L = dp.L; a.K = dp.K;
+    a.dfeat = nullptr; a.argmax = nullptr; a.accfix = nullptr; a.scale = nullptr; a.n_weights = 0; a.lambda = lambda;
     if (soft) fast_init_soft_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, stream>>>(a.ws, pairs, pd.counters);
     else fast_init_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, stream>>>(a.feat_i, pairs, pd.counters);
     count_launch();
@@ -813,14 +1074,14 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
     if (pd.n_sitems > 0) {
         const unsigned long long total = (unsigned long long)N * pd.n_sitems;
         const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms);
-        if (soft) fast_s_forward<true><<<grid, kSThreads, s_bytes, stream>>>(a);
-        else fast_s_forward<false><<<grid, kSThreads, s_bytes, stream>>>(a);
+        if (soft) fast_s_forward<1><<<grid, kSThreads, s_bytes, stream>>>(a);
+        else fast_s_forward<0><<<grid, kSThreads, s_bytes, stream>>>(a);
         count_launch();
     }
     if (fs.profile) cudaEventRecord(fs.ev[1], stream);
     if (pd.n_titems > 0) {
-        if (soft) fast_t_forward<true><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
-        else fast_t_forward<false><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
+        if (soft) fast_t_forward<1><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
+        else fast_t_forward<0><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
         count_launch();
     }
     if (fs.profile) {
@@ -833,6 +1094,72 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
         else fast_finalize_kernel<<<(unsigned)((fin + 255) / 256), 256, 0, stream>>>(feat, pd.krec, pd.n_krec, N, dp.K);
         count_launch();
     }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t n_weights, const float* X, int N,
+                                 float lambda, float shift, const float* dfeat, const int32_t* argmax, float* dW,
+                                 float* db, cudaStream_t stream) {
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = set_kernel_attributes(dev);
+    if (e != cudaSuccess) return e;
+    const size_t s_bytes = s_smem_bytes(dp.C), t_bytes = t_smem_bytes();
+    const PlanDevice& pd = fs.dev;
+    // workspace: fixed-point sums [n_weights + K], scales [K], max |x| (fixed size per handle)
+    const size_t acc_bytes = align256((size_t)(n_weights + dp.K) * 8), scale_bytes = align256((size_t)dp.K * 8);
+    if (!fs.bwd_ws) {
+        e = cudaMalloc(&fs.bwd_ws, acc_bytes + scale_bytes + 256);
+        if (e != cudaSuccess) { fs.bwd_ws = nullptr; return e; }
+    }
+    long long* accfix = static_cast<long long*>(fs.bwd_ws);
+    double* scale = reinterpret_cast<double*>(static_cast<char*>(fs.bwd_ws) + acc_bytes);
+    unsigned* absmax = reinterpret_cast<unsigned*>(static_cast<char*>(fs.bwd_ws) + acc_bytes + scale_bytes);
+    if (pd.n_titems > 0 && N > 0) {
+        e = ensure_pad_capacity(fs, N, dp.C, dp.L);
+        if (e != cudaSuccess) return e;
+    }
+    e = cudaMemsetAsync(absmax, 0, 256, stream);
+    if (e != cudaSuccess) return e;
+    const int64_t n4 = (int64_t)N * dp.C * (dp.L / 4);
+    if (n4 > 0) {
+        fast_absmax_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(X), n4, absmax);
+        count_launch();
+    }
+    fast_bwd_prepare_kernel<<<(pd.n_krec + 127) / 128, 128, 0, stream>>>(dfeat, pd.krec, pd.n_krec, N, dp.K, lambda, absmax, scale,
+                                                                         accfix, n_weights);
+    count_launch();
+    FwdArgs a;
+    a.plan = fs.dev; a.X = X; a.feat_i = nullptr; a.ws = nullptr;
+    a.c1 = lambda * 1.4426950408889634f; a.c0 = -shift * 1.4426950408889634f;
+    a.N = N; a.C = dp.C; a.L = dp.L; a.K = dp.K;
+    a.dfeat = dfeat; a.argmax = argmax; a.accfix = accfix; a.scale = scale; a.n_weights = n_weights; a.lambda = lambda;
+    if (N > 0) {
+        fast_init_kernel<<<1, 32, 0, stream>>>(nullptr, 0, pd.counters);  // resets the S work counter
+        count_launch();
+        if (pd.n_titems > 0) {
+            const int64_t rows = (int64_t)N * dp.C;
+            fast_pad_copy_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(X),
+                                                              reinterpret_cast<float4*>(fs.xpad), rows, dp.L / 4,
+                                                              fs.host.pad_pitch / 4, kTPadFront / 4);
+            count_launch();
+        }
+        if (pd.n_sitems > 0) {
+            const unsigned long long total = (unsigned long long)N * pd.n_sitems;
+            const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms);
+            fast_s_forward<2><<<grid, kSThreads, s_bytes, stream>>>(a);
+            count_launch();
+        }
+        if (pd.n_titems > 0) {
+            fast_t_forward<2><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
+            count_launch();
+        }
+    }
+    fast_bwd_finalize_kernel<<<(pd.n_krec + 127) / 128, 128, 0, stream>>>(accfix, scale, pd.krec, pd.n_krec, n_weights, dW, db);
+    count_launch();
     return cudaGetLastError();
 }
 

@@ -41,6 +41,7 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         f.nout = (int32_t)((int64_t)hp.L + 2 * (int64_t)f.p - (int64_t)(f.len - 1) * f.d);
         f.k = k; f.lo_u = -f.p; f.hi_u = f.nout - f.p;
         f.negb = 0.0f - hp.bias[k];
+        f.woff = hp.weight_offset[k];
         f.tl = (int32_t)floor_div(f.lo_u, f.d); f.rl = f.lo_u - f.tl * f.d;
         f.th = (int32_t)floor_div(f.hi_u, f.d); f.rh = f.hi_u - f.th * f.d;
         const int32_t* S = hp.channel_idx.data() + hp.channel_offset[k];
