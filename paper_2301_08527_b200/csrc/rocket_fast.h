@@ -78,17 +78,15 @@ constexpr int kTThreads = 32 * (kTConsumerWarps + 1);              // + one prod
 constexpr int kTStages = 2;
 constexpr int kTParamSlots = kTStages + 2;
 // A T tile is rg row groups x cg column groups of warp tiles, rg * cg <= 8, cg in {1, 2, 4}.
-// One box per phase brings one (cg = 1: 64 + 4 floats wide) or two (cg >= 2: 128 + 4 wide)
-// column groups; cg = 4 takes two boxes per phase.
-ROCKET_CX int t_box_cols(int cg) { return cg == 1 ? kWarpCols + 4 : 2 * kWarpCols + 4; }
-ROCKET_CX int t_boxes_per_phase(int cg) { return cg <= 2 ? 1 : 2; }
-// Box rows of one phase (rows s, s+4, ..), and the phase pitch in floats (a multiple of 32
-// floats keeps every box destination 128-byte aligned).
+// One box per phase brings all column groups (64 * cg floats wide).  The zero-margined copy is kept
+// four times, shifted by 0, 1, 2 and 3 floats, so that every row start is 16-byte aligned in one
+// of them: a box needs no alignment slack and every pair a consumer reads is 8-byte aligned.
+ROCKET_CX int t_box_cols(int cg) { return kWarpCols * cg; }
+// Box rows of one phase (rows s, s+4, ..), and the floats of one phase box (a multiple of 64
+// floats, so every box destination stays 128-byte aligned).
 ROCKET_CX int t_box_rows(int rg, int len) { return (kR * rg + len - 1 + 3) / 4; }
-ROCKET_CX int t_phase_floats(int cg, int box_rows) { return (box_rows * t_box_cols(cg) + 31) / 32 * 32; }
-ROCKET_CX int t_stage_floats(int rg, int cg, int len) {
-    return 4 * t_boxes_per_phase(cg) * t_phase_floats(cg, t_box_rows(rg, len));
-}
+ROCKET_CX int t_phase_floats(int cg, int box_rows) { return box_rows * t_box_cols(cg); }
+ROCKET_CX int t_stage_floats(int rg, int cg, int len) { return 4 * t_phase_floats(cg, t_box_rows(rg, len)); }
 ROCKET_CX int imax_cx(int a, int b) { return a > b ? a : b; }
 constexpr int kTStageFloats = imax_cx(imax_cx(t_stage_floats(8, 1, ROCKET_MAX_LENGTH), t_stage_floats(4, 2, ROCKET_MAX_LENGTH)),
                                       t_stage_floats(2, 4, ROCKET_MAX_LENGTH));
@@ -103,7 +101,8 @@ struct alignas(16) TItem {
     int32_t krec;                         // index into the kernel records
     int32_t cg, pad0_[3];
     int32_t x[4], y[4];                   // tensor coordinates of the four phase boxes
-    int32_t pad1_[8];
+    int32_t j[4];                         // which shifted copy each phase reads
+    int32_t pad1_[4];
 };
 static_assert(sizeof(TItem) == 128, "TItem must be 32 words");
 // One tensor map: boxes of box_cols x box_rows floats over runs of 4 * d floats.
@@ -147,8 +146,9 @@ struct FastState {
     PlanDevice dev;
     void* plan_blob = nullptr;            // records, buckets, items, counters, error flag
     void* maps_blob = nullptr;            // tensor maps
-    float* xpad = nullptr;                // padded copy, capacity pad_examples
+    float* xpad = nullptr;                // the four shifted zero-margined copies, capacity pad_examples
     int pad_examples = 0;
+    int64_t copy_floats = 0;              // floats of one copy
     void* soft_ws = nullptr;              // soft mode: 16 bytes per (example, kernel), grows with N
     size_t soft_ws_bytes = 0;
     void* bwd_ws = nullptr;               // backward: fixed-point sums [n_weights + K], scales [K], max |x|

@@ -60,8 +60,8 @@ __device__ __forceinline__ float key_float(int k) { return __int_as_float(k >= 0
 
 // One channel of one warp tile: 16 output rows of the thread's column pair, 16+ELL-1 input pairs
 // streamed past them.  Row s of the tile sits at st[off[s & 3] + (s >> 2) * STEP]; w2 holds the
-// channel's negated weights, each twice.  With ODD, rows of odd s are only 4-byte aligned.
-template <int ELL, bool ODD, int STEP>
+// channel's negated weights, each twice.
+template <int ELL, int STEP>
 __device__ __forceinline__ void conv_channel(const float* __restrict__ st, const int (&off)[4],
                                              const float* __restrict__ w2, u64 (&acc)[kR]) {
     u64 wp[ELL + 1];
@@ -74,9 +74,7 @@ __device__ __forceinline__ void conv_channel(const float* __restrict__ st, const
 #pragma unroll
     for (int s = 0; s < kR + ELL - 1; ++s) {
         const float* p = st + off[s & 3] + (s >> 2) * STEP;
-        u64 x;
-        if (ODD && (s & 1)) x = pack2(p[0], p[1]);
-        else x = *reinterpret_cast<const u64*>(p);
+        const u64 x = *reinterpret_cast<const u64*>(p);
 #pragma unroll
         for (int j = 0; j < ELL; ++j) {
             const int o = s - j;
@@ -242,15 +240,13 @@ __device__ __forceinline__ float make_gz(u64 (&acc)[kR], float c1, float c0, flo
 
 // Backward, second half, one channel of one warp tile: dw[j] += gz[o] * x[o + j] for the thread's
 // column pair (same traversal as conv_channel with the roles of weights and accumulators swapped).
-template <int ELL, bool ODD, int STEP>
+template <int ELL, int STEP>
 __device__ __forceinline__ void grad_channel(const float* __restrict__ st, const int (&off)[4], const u64 (&gz)[kR],
                                              u64 (&dw)[ELL]) {
 #pragma unroll
     for (int s = 0; s < kR + ELL - 1; ++s) {
         const float* p = st + off[s & 3] + (s >> 2) * STEP;
-        u64 x;
-        if (ODD && (s & 1)) x = pack2(p[0], p[1]);
-        else x = *reinterpret_cast<const u64*>(p);
+        const u64 x = *reinterpret_cast<const u64*>(p);
 #pragma unroll
         for (int j = 0; j < ELL; ++j) {
             const int o = s - j;
@@ -336,7 +332,7 @@ __device__ __forceinline__ void s_grad_tile(const float* planes, const KRec* rec
         u64 dw[ELL];
 #pragma unroll
         for (int j = 0; j < ELL; ++j) dw[j] = 0ull;
-        grad_channel<ELL, false, 4 * kWarpCols>(planes + rec->ch[q] * kSPlaneFloats, off, gz, dw);
+        grad_channel<ELL, 4 * kWarpCols>(planes + rec->ch[q] * kSPlaneFloats, off, gz, dw);
         reduce_publish_dw<ELL>(dw, accfix + rec->woff + q * ELL, scale, lane);
     }
 }
@@ -346,7 +342,7 @@ __device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* r
     const int m = rec->m;
     const int off[4] = {2 * lane, kWarpCols + 2 * lane, 2 * kWarpCols + 2 * lane, 3 * kWarpCols + 2 * lane};
     for (int q = 0; q < m; ++q)
-        conv_channel<ELL, false, 4 * kWarpCols>(planes + rec->ch[q] * kSPlaneFloats, off, rec->w2[q], acc);
+        conv_channel<ELL, 4 * kWarpCols>(planes + rec->ch[q] * kSPlaneFloats, off, rec->w2[q], acc);
 }
 
 template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft
@@ -506,11 +502,11 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-// Tiled TMA load of one 3-D box (x a multiple of 4 floats), completion on bar.
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, int x, int y, int z, uint32_t bar) {
+// Tiled TMA load of one 4-D box (x a multiple of 4 floats), completion on bar.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, int x, int y, int z, int w, uint32_t bar) {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar) : "memory");
 }
 
 // What the producer tells the consumers about a tile (written with plain stores before its
@@ -528,14 +524,14 @@ struct TShared {
 
 // The channels of one tile for one consumer warp; returns false when a wait gave up.  A warp
 // without a valid output (active == false) only keeps the ring moving.
-template <int ELL, bool ODD, int STEP>
+template <int ELL, int STEP>
 __device__ __forceinline__ bool t_channels(const float* stages, const KRec* rec, const int (&off)[4], uint32_t full0,
                                            uint32_t empty0, uint32_t& st, int lane, bool active, u64 (&acc)[kR]) {
     const int m = rec->m;
     for (int q = 0; q < m; ++q) {
         const uint32_t slot = st % kTStages;
         if (q > 0 && !mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) return false;
-        if (active) conv_channel<ELL, ODD, STEP>(stages + slot * kTStageFloats, off, rec->w2[q], acc);
+        if (active) conv_channel<ELL, STEP>(stages + slot * kTStageFloats, off, rec->w2[q], acc);
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * slot);
         ++st;
@@ -544,7 +540,7 @@ __device__ __forceinline__ bool t_channels(const float* stages, const KRec* rec,
 }
 
 // Backward second half on a T tile: the kernel's channels stream through the ring once more.
-template <int ELL, bool ODD, int STEP>
+template <int ELL, int STEP>
 __device__ __forceinline__ bool t_grad_channels(const float* stages, const KRec* rec, const int (&off)[4], uint32_t full0,
                                                 uint32_t empty0, uint32_t& st, int lane, bool active, const u64 (&gz)[kR],
                                                 long long* accfix, double scale) {
@@ -556,7 +552,7 @@ __device__ __forceinline__ bool t_grad_channels(const float* stages, const KRec*
             u64 dw[ELL];
 #pragma unroll
             for (int j = 0; j < ELL; ++j) dw[j] = 0ull;
-            grad_channel<ELL, ODD, STEP>(stages + slot * kTStageFloats, off, gz, dw);
+            grad_channel<ELL, STEP>(stages + slot * kTStageFloats, off, gz, dw);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + 8u * slot);
             reduce_publish_dw<ELL>(dw, accfix + rec->woff + q * ELL, scale, lane);
@@ -570,27 +566,21 @@ __device__ __forceinline__ bool t_grad_channels(const float* stages, const KRec*
 }
 
 template <int STEP>
-__device__ __forceinline__ bool t_grad_dispatch(int len, bool odd, const float* stages, const KRec* rec, const int (&off)[4],
+__device__ __forceinline__ bool t_grad_dispatch(int len, const float* stages, const KRec* rec, const int (&off)[4],
                                                 uint32_t full0, uint32_t empty0, uint32_t& st, int lane, bool active,
                                                 const u64 (&gz)[kR], long long* accfix, double scale) {
-    if (len == 7) return odd ? t_grad_channels<7, true, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale)
-                             : t_grad_channels<7, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale);
-    if (len == 9) return odd ? t_grad_channels<9, true, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale)
-                             : t_grad_channels<9, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale);
-    return odd ? t_grad_channels<11, true, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale)
-               : t_grad_channels<11, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale);
+    if (len == 7) return t_grad_channels<7, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale);
+    if (len == 9) return t_grad_channels<9, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale);
+    return t_grad_channels<11, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale);
 }
 
 template <int STEP>
-__device__ __forceinline__ bool t_dispatch(int len, bool odd, const float* stages, const KRec* rec, const int (&off)[4],
+__device__ __forceinline__ bool t_dispatch(int len, const float* stages, const KRec* rec, const int (&off)[4],
                                            uint32_t full0, uint32_t empty0, uint32_t& st, int lane, bool active,
                                            u64 (&acc)[kR]) {
-    if (len == 7) return odd ? t_channels<7, true, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc)
-                             : t_channels<7, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
-    if (len == 9) return odd ? t_channels<9, true, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc)
-                             : t_channels<9, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
-    return odd ? t_channels<11, true, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc)
-               : t_channels<11, false, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
+    if (len == 7) return t_channels<7, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
+    if (len == 9) return t_channels<9, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
+    return t_channels<11, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
 }
 
 template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft
@@ -625,22 +615,21 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
             bool ok = true;
             const int4* tp = reinterpret_cast<const int4*>(a.plan.titems + i_beg);
             int4 w0 = __ldg(tp), w1 = __ldg(tp + 1), w2 = __ldg(tp + 2), w3 = __ldg(tp + 3), w4 = __ldg(tp + 4),
-                 w5 = __ldg(tp + 5);
+                 w5 = __ldg(tp + 5), w6 = __ldg(tp + 6);
             for (int n = 0; ok && n < a.N; ++n) {
                 for (int i = i_beg; ok && i < i_end; ++i) {
                     if (*abort_flag) { ok = false; break; }
                     const int map = w0.x, t0 = w0.y, r0 = w0.z, rg = w0.w;
                     const int m = w1.z, box_rows = w1.w, krec = w2.w, cg = w3.x;
                     const unsigned chw[3] = {(unsigned)w2.x, (unsigned)w2.y, (unsigned)w2.z};
-                    const int px[4] = {w4.x, w4.y, w4.z, w4.w}, py[4] = {w5.x, w5.y, w5.z, w5.w};
+                    const int px[4] = {w4.x, w4.y, w4.z, w4.w}, py[4] = {w5.x, w5.y, w5.z, w5.w}, pj[4] = {w6.x, w6.y, w6.z, w6.w};
                     {   // the next tile's description is on its way while this one is issued
                         int inext = i + 1;
                         if (inext == i_end) inext = i_beg;
                         tp = reinterpret_cast<const int4*>(a.plan.titems + inext);
                         w0 = __ldg(tp); w1 = __ldg(tp + 1); w2 = __ldg(tp + 2); w3 = __ldg(tp + 3); w4 = __ldg(tp + 4);
-                        w5 = __ldg(tp + 5);
+                        w5 = __ldg(tp + 5); w6 = __ldg(tp + 6);
                     }
-                    const int nbx = t_boxes_per_phase(cg);
                     const uint32_t box_bytes = (uint32_t)box_rows * (uint32_t)t_box_cols(cg) * 4u;
                     const uint32_t phase_bytes = (uint32_t)t_phase_floats(cg, box_rows) * 4u;
                     const char* tmap = reinterpret_cast<const char*>(a.plan.tmaps) + (size_t)map * 128;
@@ -656,7 +645,7 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                             break;
                         }
                         const uint32_t bar = full0 + 8u * slot;
-                        uint32_t tx = (uint32_t)nbx * 4u * box_bytes;
+                        uint32_t tx = 4u * box_bytes;
                         if (q2 == 0) {
                             TSlotItem& si = sh.items[it % kTParamSlots];
                             si.t0 = t0; si.r0 = r0; si.rg = rg; si.cg = cg; si.box_rows = box_rows; si.rec_slot = (int)rslot;
@@ -667,11 +656,8 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                         const int ch = (int)((chw[q >> 2] >> (8 * (q & 3))) & 0xffu);
                         const int z = n * a.C + ch;
                         const uint32_t dst0 = smem_u32(stages + slot * kTStageFloats);
-                        for (int bx = 0; bx < nbx; ++bx)
 #pragma unroll
-                            for (int k = 0; k < 4; ++k)
-                                tma_load_3d(dst0 + (uint32_t)(bx * 4 + k) * phase_bytes, tmap, px[k] + 2 * kWarpCols * bx, py[k], z,
-                                            bar);
+                        for (int k = 0; k < 4; ++k) tma_load_4d(dst0 + (uint32_t)k * phase_bytes, tmap, px[k], py[k], z, pj[k], bar);
                         ++st;
                     }
                     ++it;
@@ -713,17 +699,15 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                 valid_rows_tc(t0 + kR * wr, r0 + lc + 1, rec->tl, rec->rl, rec->th, rec->rh, kR, ok1, lo1, hi1);
                 const bool interior = __all_sync(kFull, lo0 == 0 && lo1 == 0 && hi0 == kR && hi1 == kR);
                 const bool active = __any_sync(kFull, lo0 < hi0 || lo1 < hi1);
-                const int bx = cg == 1 ? 0 : wc >> 1, incol = cg == 1 ? 0 : (wc & 1) * kWarpCols;
                 const int boxw = t_box_cols(cg);
                 int off[4];
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    off[k] = t_box_offset(cg, bx, k, box_rows) + 4 * wr * boxw + (((t0 + k) * d) & 3) + incol + 2 * lane;
+                for (int k = 0; k < 4; ++k) off[k] = t_box_offset(cg, k, box_rows) + 4 * wr * boxw + lc;
                 u64 acc[kR];
                 init_acc(acc, rec->negb, interior, lo0, hi0, lo1, hi1);
-                const bool odd = (d & 1) != 0;
-                if (cg == 1) ok = t_dispatch<kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
-                else ok = t_dispatch<2 * kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc);
+                if (cg == 1) ok = t_dispatch<kWarpCols>(len, stages, rec, off, full0, empty0, st, lane, active, acc);
+                else if (cg == 2) ok = t_dispatch<2 * kWarpCols>(len, stages, rec, off, full0, empty0, st, lane, active, acc);
+                else ok = t_dispatch<4 * kWarpCols>(len, stages, rec, off, full0, empty0, st, lane, active, acc);
                 if (!ok) break;
                 if (MODE == 2) {
                     const int64_t pair = (int64_t)n * a.K + korig;
@@ -743,10 +727,9 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                         scale = __ldg(a.scale + korig);
                         if (lane == 0) add_fixed(a.accfix + a.n_weights + korig, dbs, scale);
                     }
-                    if (cg == 1) ok = t_grad_dispatch<kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc,
-                                                                     a.accfix, scale);
-                    else ok = t_grad_dispatch<2 * kWarpCols + 4>(len, odd, stages, rec, off, full0, empty0, st, lane, active, acc,
-                                                                 a.accfix, scale);
+                    if (cg == 1) ok = t_grad_dispatch<kWarpCols>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale);
+                    else if (cg == 2) ok = t_grad_dispatch<2 * kWarpCols>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale);
+                    else ok = t_grad_dispatch<4 * kWarpCols>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale);
                     if (!ok) break;
                 } else if (active) {
                     if (MODE == 1) {
@@ -774,13 +757,22 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
 // ------------------------------------------------------------------------------------------------
 // pad copy / init / finalise
 // ------------------------------------------------------------------------------------------------
-__global__ void fast_pad_copy_kernel(const float4* __restrict__ X, float4* __restrict__ xpad, int64_t rows, int L4,
-                                     int64_t pitch4, int front4) {
+// Writes the samples of the batch into the four shifted copies: copy j holds the zero-margined
+// layout moved down by j floats (copy_j[i] = layout[i + j]); margins are never written and stay zero.
+__global__ void fast_pad_copy_kernel(const float4* __restrict__ X, float* __restrict__ xpad, int64_t rows, int L4,
+                                     int64_t pitch, int front, int64_t copy_floats) {
     const int64_t total = rows * L4;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
         const int64_t rho = e / L4;
         const int i = (int)(e - rho * L4);
-        xpad[rho * pitch4 + front4 + i] = __ldg(X + e);
+        const float4 v = __ldg(X + e);
+        float* dst = xpad + rho * pitch + front + 4 * (int64_t)i;
+        *reinterpret_cast<float4*>(dst) = v;
+#pragma unroll
+        for (int j = 1; j < 4; ++j) {
+            float* dj = dst + j * copy_floats - j;
+            dj[0] = v.x; dj[1] = v.y; dj[2] = v.z; dj[3] = v.w;
+        }
     }
 }
 
@@ -991,7 +983,8 @@ cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L) {
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
     const int64_t pitch = fs.host.pad_pitch, rows = (int64_t)N * C;
-    const size_t bytes = (size_t)(rows + 1) * (size_t)pitch * 4;
+    const int64_t copy_floats = (rows + 1) * pitch;   // pitch is a multiple of 32 floats
+    const size_t bytes = (size_t)copy_floats * 4 * 4;
     if (fs.xpad) cudaFree(fs.xpad);  // waits for work that still reads it
     fs.xpad = nullptr;
     fs.pad_examples = 0;
@@ -1004,11 +997,11 @@ cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L) {
     for (size_t i = 0; i < n_maps; ++i) {
         const TMapSpec& sp = fs.host.tmaps[i];
         const cuuint64_t run = 4ull * (cuuint64_t)sp.d;
-        const cuuint64_t dims[3] = {run + kTXExtra, ((cuuint64_t)kTPadFront + (cuuint64_t)L + run - 1) / run, (cuuint64_t)rows};
-        const cuuint64_t strides[2] = {run * 4ull, (cuuint64_t)pitch * 4ull};
-        const cuuint32_t box[3] = {(cuuint32_t)sp.box_cols, (cuuint32_t)sp.box_rows, 1u};
-        const cuuint32_t elem[3] = {1u, 1u, 1u};
-        const CUresult r = encode(&maps[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, fs.xpad, dims, strides, box, elem,
+        const cuuint64_t dims[4] = {run + kTXExtra, ((cuuint64_t)kTPadFront + (cuuint64_t)L + run - 1) / run, (cuuint64_t)rows, 4ull};
+        const cuuint64_t strides[3] = {run * 4ull, (cuuint64_t)pitch * 4ull, (cuuint64_t)copy_floats * 4ull};
+        const cuuint32_t box[4] = {(cuuint32_t)sp.box_cols, (cuuint32_t)sp.box_rows, 1u, 1u};
+        const cuuint32_t elem[4] = {1u, 1u, 1u, 1u};
+        const CUresult r = encode(&maps[i], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, fs.xpad, dims, strides, box, elem,
                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
@@ -1021,6 +1014,7 @@ cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L) {
     e = cudaMemcpy(fs.maps_blob, maps.data(), n_maps * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
     if (e != cudaSuccess) return e;
     fs.pad_examples = N;
+    fs.copy_floats = copy_floats;
     fs.dev.tmaps = fs.maps_blob;
     fs.dev.xpad = fs.xpad;
     return cudaSuccess;
@@ -1062,8 +1056,8 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
     if (pd.n_titems > 0) {
         const int64_t rows = (int64_t)N * dp.C;
         fast_pad_copy_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(X),
-                                                          reinterpret_cast<float4*>(fs.xpad), rows, dp.L / 4,
-                                                          fs.host.pad_pitch / 4, kTPadFront / 4);
+                                                          fs.xpad, rows, dp.L / 4, fs.host.pad_pitch, kTPadFront,
+                                                          fs.copy_floats);
         count_launch();
     }
     if (fs.profile) {
@@ -1143,8 +1137,8 @@ cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t 
         if (pd.n_titems > 0) {
             const int64_t rows = (int64_t)N * dp.C;
             fast_pad_copy_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(X),
-                                                              reinterpret_cast<float4*>(fs.xpad), rows, dp.L / 4,
-                                                              fs.host.pad_pitch / 4, kTPadFront / 4);
+                                                              fs.xpad, rows, dp.L / 4, fs.host.pad_pitch,
+                                                              kTPadFront, fs.copy_floats);
             count_launch();
         }
         if (pd.n_sitems > 0) {

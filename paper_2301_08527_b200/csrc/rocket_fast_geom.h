@@ -43,32 +43,29 @@ ROCKET_HD int s_column_u0(const SBucket& b, int cg) {
 // T regime.  A tile starts at A-row t0 and residue r0 (a multiple of 64).  Row s of the tile
 // (A-row t0 + s) arrives with the box of phase s & 3, as that box's row s >> 2.  In the
 // zero-margined copy the element (A-row t, residue r) of a channel row sits at float
-// front + t*d + r of that row; the copy is seen as runs of 4d floats (tensor coordinate y = which
-// run, x = position in the run).  A box starts at the 16-byte aligned x just below the element
-// it wants, which then sits `shift` floats into the box row.
-struct TPhase { int x, y, shift; };
+// front + t*d + r of that row; copy j holds the same data moved down by j floats, so the element
+// is 16-byte aligned in copy j = position & 3.  Every copy is seen as runs of 4d floats (tensor
+// coordinate y = which run, x = position in the run).
+struct TPhase { int x, y, j; };
 
 ROCKET_HD TPhase t_phase(int t0, int r0, int d, int k) {
     const long long flat = (long long)kTPadFront + (long long)(t0 + k) * d + r0;
-    const long long run = 4ll * d;
-    long long y = flat / run;
-    if (flat - y * run < 0) --y;  // floor for negative positions
-    const int x = (int)(flat - y * run);
     TPhase p;
-    p.shift = x & 3;
-    p.x = x - p.shift;
+    p.j = (int)(flat & 3);
+    const long long pos = flat - p.j, run = 4ll * d;
+    long long y = pos / run;
+    if (pos - y * run < 0) --y;  // floor for negative positions
+    p.x = (int)(pos - y * run);
     p.y = (int)y;
     return p;
 }
 
-// Float offset, inside a stage, of box bx (0 or 1) of phase k.
-ROCKET_HD int t_box_offset(int cg, int bx, int k, int box_rows) { return (bx * 4 + k) * t_phase_floats(cg, box_rows); }
+// Float offset, inside a stage, of the box of phase k.
+ROCKET_HD int t_box_offset(int cg, int k, int box_rows) { return k * t_phase_floats(cg, box_rows); }
 
 // Float offset, inside a stage, of tile row s / tile column lc as the consumer reads it.
-ROCKET_HD int t_elem_offset(int cg, int s, int lc, int box_rows, int shift) {
-    const int wc = lc >> 6;
-    const int bx = cg == 1 ? 0 : wc >> 1, incol = cg == 1 ? 0 : (wc & 1) * kWarpCols;
-    return t_box_offset(cg, bx, s & 3, box_rows) + (s >> 2) * t_box_cols(cg) + shift + incol + (lc & 63);
+ROCKET_HD int t_elem_offset(int cg, int s, int lc, int box_rows) {
+    return t_box_offset(cg, s & 3, box_rows) + (s >> 2) * t_box_cols(cg) + lc;
 }
 
 }  // namespace fast

@@ -108,10 +108,8 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         const KRec f = out.krec.back();
         out.flops_t += 2.0 * f.len * f.m * (double)f.nout;
         d_max = std::max(d_max, f.d);
-        int64_t tmin = floor_div(f.lo_u, f.d);
+        const int64_t tmin = floor_div(f.lo_u, f.d);
         const int64_t tmax = floor_div((int64_t)f.hi_u - 1, f.d);
-        // odd dilations: an even first row keeps the rows of phases 0 and 2 aligned to pairs
-        if (f.d & 1) tmin = floor_div(tmin, 2) * 2;
         const int R16 = (int)((tmax - tmin + 1 + kR - 1) / kR), C64 = (f.d + kWarpCols - 1) / kWarpCols;
         // column chunks for a main width cg: C64 / cg chunks of cg, the rest in chunks of 2 and 1
         auto chunks_of = [&](int cg, std::vector<int>& widths) {
@@ -150,7 +148,7 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
                 it.map = found->second;
                 for (int ph = 0; ph < 4; ++ph) {
                     const TPhase tp = t_phase(it.t0, it.r0, it.d, ph);
-                    it.x[ph] = tp.x; it.y[ph] = tp.y;
+                    it.x[ph] = tp.x; it.y[ph] = tp.y; it.j[ph] = tp.j;
                 }
                 out.tcost.push_back((double)f.m * (f.len + 2) + 8.0);
                 out.titems.push_back(it);
@@ -160,7 +158,7 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
     }
     // every channel row of the zero-margined copy: front zeros, L samples, zeros for the run a box may
     // read past the last sample; rounded to 128 bytes
-    const int64_t pitch = (int64_t)kTPadFront + hp.L + 4ll * d_max + kTXExtra + t_box_cols(2);
+    const int64_t pitch = (int64_t)kTPadFront + hp.L + 4ll * d_max + kTXExtra + t_box_cols(4);
     out.pad_pitch = (pitch + 31) / 32 * 32;
 }
 

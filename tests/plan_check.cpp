@@ -88,32 +88,29 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
         REQUIRE(f.d >= kTMinDilation && f.d == it.d && f.len == it.len && f.m == it.m, "T item fields");
         REQUIRE((it.cg == 1 || it.cg == 2 || it.cg == 4) && it.rg >= 1 && it.rg * it.cg <= kTConsumerWarps, "T shape");
         REQUIRE(it.r0 % kWarpCols == 0 && it.r0 < f.d, "T column origin");
-        REQUIRE(!(f.d & 1) || (it.t0 % 2 == 0), "odd dilation needs an even first row");
         for (int q = 0; q < f.m; ++q) REQUIRE(it.ch[q] == f.ch[q], "T channel list");
-        const int rows_out = kR * it.rg, groups = it.cg, boxw = t_box_cols(it.cg), nbx = t_boxes_per_phase(it.cg);
+        const int rows_out = kR * it.rg, groups = it.cg, boxw = t_box_cols(it.cg);
         const int rows = rows_out + f.len - 1;
         REQUIRE(it.box_rows == t_box_rows(it.rg, f.len) && 4 * it.box_rows >= rows, "T box rows");
         REQUIRE(sp.d == f.d && sp.box_cols == boxw && sp.box_rows == it.box_rows && boxw <= 256 && it.box_rows <= 256, "T map spec");
-        REQUIRE(4 * nbx * t_phase_floats(it.cg, it.box_rows) <= kTStageFloats, "stage size");
+        REQUIRE(4 * t_phase_floats(it.cg, it.box_rows) <= kTStageFloats, "stage size");
         const long long run = 4ll * f.d, ny = (kTPadFront + (long long)L + run - 1) / run;
         // the boxes the producer issues
         TPhase ph[4];
         for (int k = 0; k < 4; ++k) {
             ph[k] = t_phase(it.t0, it.r0, f.d, k);
-            REQUIRE(ph[k].x % 4 == 0 && ph[k].x >= 0 && ph[k].x < run, "box x");
-            REQUIRE(it.x[k] == ph[k].x && it.y[k] == ph[k].y, "stored box coordinates");
-            for (int bx = 0; bx < nbx; ++bx) {
-                const int x = ph[k].x + 2 * kWarpCols * bx;
-                REQUIRE(x + boxw <= run + kTXExtra, "box leaves the tensor row");
-                const int dst = t_box_offset(it.cg, bx, k, it.box_rows);
-                REQUIRE(dst % 32 == 0 && dst + it.box_rows * boxw <= kTStageFloats, "box destination");
-                for (int j = 0; j < it.box_rows; ++j) {
-                    const long long y = ph[k].y + j;
-                    if (y < 0 || y >= ny) continue;  // zero-filled by the copy engine
-                    const long long first = y * run + x, last = first + boxw - 1;
-                    REQUIRE(first >= 0 && last < pitch, "box row reads outside its channel row: %lld..%lld of %lld", first,
-                            last, (long long)pitch);
-                }
+            REQUIRE(ph[k].x % 4 == 0 && ph[k].x >= 0 && ph[k].x < run && ph[k].j >= 0 && ph[k].j < 4, "box x");
+            REQUIRE(it.x[k] == ph[k].x && it.y[k] == ph[k].y && it.j[k] == ph[k].j, "stored box coordinates");
+            REQUIRE(ph[k].x + boxw <= run + kTXExtra, "box leaves the tensor row");
+            const int dst = t_box_offset(it.cg, k, it.box_rows);
+            REQUIRE(dst % 32 == 0 && dst + it.box_rows * boxw <= kTStageFloats, "box destination");
+            for (int j = 0; j < it.box_rows; ++j) {
+                const long long y = ph[k].y + j;
+                if (y < 0 || y >= ny) continue;  // zero-filled by the copy engine
+                // copy j holds the layout moved down by j floats: the box row reads layout[first + j .. last + j]
+                const long long first = y * run + ph[k].x + ph[k].j, last = first + boxw - 1;
+                REQUIRE(first >= 0 && last < pitch, "box row reads outside its channel row: %lld..%lld of %lld", first,
+                        last, (long long)pitch);
             }
         }
         // what every consumer thread owns and reads
@@ -133,18 +130,15 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
                 if (o_lo >= o_hi) continue;
                 for (int s2 = 0; s2 < kR + f.len - 1; ++s2) {
                     const int s = kR * wr + s2, k = s & 3;
-                    const int shift = ((it.t0 + k) * f.d) & 3;
-                    REQUIRE(shift == ph[k].shift, "alignment shift");
-                    const int pos = t_elem_offset(it.cg, s, lc, it.box_rows, shift);
+                    const int pos = t_elem_offset(it.cg, s, lc, it.box_rows);
                     REQUIRE(pos >= 0 && pos < kTStageFloats, "read outside the stage");
-                    if ((lc & 1) == 0) REQUIRE(((f.d & 1) && (s2 & 1)) || pos % 2 == 0, "pair not 8-byte aligned");
+                    if ((lc & 1) == 0) REQUIRE(pos % 2 == 0, "pair not 8-byte aligned");
                     // which sample the copy engine put there
-                    const int wc = lc >> 6, bx = it.cg == 1 ? 0 : wc >> 1;
-                    const int rel = pos - t_box_offset(it.cg, bx, k, it.box_rows);
+                    const int rel = pos - t_box_offset(it.cg, k, it.box_rows);
                     const int j = rel / boxw, i = rel % boxw;
                     REQUIRE(rel >= 0 && j < it.box_rows, "read outside the box");
                     const long long y = ph[k].y + j;
-                    const long long flat = y * run + ph[k].x + 2 * kWarpCols * bx + i;
+                    const long long flat = y * run + ph[k].x + i + ph[k].j;
                     const long long want = (long long)kTPadFront + (long long)(it.t0 + s) * f.d + it.r0 + lc;
                     REQUIRE(flat == want, "wrong sample: got flat %lld, want %lld", flat, want);
                     const bool in_series = want >= kTPadFront && want < kTPadFront + L;
