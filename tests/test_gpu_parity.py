@@ -186,6 +186,56 @@ def test_config3_training_pass_sampled(path):
         P.check_grads(dW, db, rdW, rdb)
 
 
+
+def test_config3_full_kernel_set_soft_and_backward_sampled():
+    # N=32 x C=20 x L=50,000 with all 10,000 kernels through the automatic path, as bench.py times it;
+    # the oracle checks a sample: soft features and argmax on random pairs, gradients on a few kernels
+    # over the whole batch (a kernel's gradient does not depend on the other kernels).
+    torch = _torch()
+    N, K, C, L, lam, shift = 32, 10000, 20, 50000, 10.0, 3.0
+    kp = generate_kernels(8527, K, C, L)
+    X = ar1_spike_series(2301, N, C, L)
+    g = normal_array(527, (N, 2 * K))
+    p = rk.RocketParams.from_kernel_params(kp)
+    Xd = _dev(X)
+    feat, arg = rk.rocket_transform_soft(p, Xd, lam, shift)
+    feat, arg = feat.cpu().numpy(), arg.cpu().numpy()
+    assert p.device_status() == 0
+    assert np.all(np.isfinite(feat)) and np.all((feat[:, 0::2] >= 0) & (feat[:, 0::2] <= 1))   # fp32 may round to the ends
+    rng = np.random.default_rng(4)
+    pn = rng.integers(0, N, 500).astype(np.int32)
+    pk = rng.integers(0, K, 500).astype(np.int32)
+    _check_sampled(kp, X, feat, pn, pk, soft=(lam, shift), arg=arg)
+    # gradients of 10 kernels over the whole batch; the oracle's argmax feeds both sides
+    ks = np.sort(rng.choice(K, 10, replace=False)).astype(np.int32)
+    ref = oracle.forward_pairs(kp, X, np.repeat(np.arange(N), len(ks)).astype(np.int32), np.tile(ks, N), lam=lam, shift=shift)
+    arg_in = arg.copy()
+    arg_in[:, ks] = ref.argmax.reshape(N, len(ks))
+    dW, db = rk.rocket_transform_soft_backward(p, Xd, lam, shift, _dev(g), _dev(arg_in.astype(np.int32)))
+    dW, db = dW.cpu().numpy(), db.cpu().numpy()
+    assert p.device_status() == 0
+    p.close()
+    rdW, rdb = oracle.backward(kp, X, g, arg_in, lam=lam, shift=shift, kernels=ks)
+    sel = np.concatenate([np.arange(kp.weight_offset[k], kp.weight_offset[k + 1]) for k in ks])
+    P.check_grads(dW[sel], db[ks], rdW[sel], rdb[ks])
+    assert np.all(np.isfinite(dW)) and np.all(np.isfinite(db))
+
+
+@pytest.mark.parametrize("N,L,K", [(1, 10000, 10000), (8, 200000, 10000), (256, 10000, 50000), (60, 50000, 50000)])
+def test_config4_sweep_points_hard_sampled(N, L, K):
+    # corners of the throughput sweep (batch 1 = streaming latency, the longest series, the largest batch,
+    # the largest kernel set); the oracle checks a sample of pairs, the rest is covered by invariants
+    kp = generate_kernels(8527, K, 20, L)
+    X = ar1_spike_series(2301, N, 20, L)
+    feat = _run_hard(kp, X, 0)
+    _check_properties_hard(feat)
+    rng = np.random.default_rng(N + L + K)
+    n_pairs = 300 if L <= 50000 else 120
+    pn = rng.integers(0, N, n_pairs).astype(np.int32)
+    pk = rng.integers(0, K, n_pairs).astype(np.int32)
+    _check_sampled(kp, X, feat, pn, pk)
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_edge_cases(path):
     torch = _torch()
