@@ -167,6 +167,7 @@ def main():
     ap.add_argument("--ref-kernels", type=int, default=2000, help="kernels per step of the reference arm's sample")
     ap.add_argument("--skip-passes", action="store_true", help="skip the soft forward / backward timings")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="also time the throughput sweep (config 4) on rank 0")
     ap.add_argument("--small", action="store_true", help="profiling case: N=8 examples (160 MB... of input)")
     args = ap.parse_args()
 
@@ -318,6 +319,26 @@ def main():
                               "flop_count": "4*len*channels*L_out (recompute z + dW)"},
         }
 
+    sweep = None
+    if args.sweep and rank == 0:
+        # config 4: hard transform, N in {1, 8, 60, 256} x L in {10k, 50k, 200k} x K in {10k, 50k}; N = 1 is the
+        # streaming latency.  Fresh inputs per (N, L); three timed calls after two warm-ups.
+        sweep = []
+        for L4 in (10000, 50000, 200000):
+            for K4 in (10000, 50000):
+                p4 = rk.RocketParams.generate(PARAM_SEED, K4, 20, L4)
+                fl4, _ = p4.work()
+                for N4 in (1, 8, 60, 256):
+                    X4 = torch.from_numpy(ar1_spike_series(DATA_SEED, min(N4, 8), 20, L4)).cuda()
+                    X4 = X4.repeat((N4 + X4.shape[0] - 1) // X4.shape[0], 1, 1)[:N4].contiguous()
+                    f4 = torch.empty((N4, 2 * K4), dtype=torch.float32, device="cuda")
+                    t4, _ = time_steps(lambda: rk.rocket_transform(p4, X4, out=f4), 3, 2)
+                    t4 /= 3
+                    sweep.append({"N": N4, "L": L4, "K": K4, "ms": 1e3 * t4, "examples_per_s": N4 / t4,
+                                  "conv_tflops": fl4 * N4 / t4 / 1e12})
+                    del X4, f4
+                p4.close()
+
     cpu = None
     if rank == 0 and world == 1 and not args.skip_cpu_baseline:
         kp = generate_kernels(PARAM_SEED, w["K"], w["C"], w["L"])
@@ -337,6 +358,8 @@ def main():
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_timed,
             "clocks": clocks, "passes": passes,
         }
+        if sweep is not None:
+            line["sweep"] = sweep
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

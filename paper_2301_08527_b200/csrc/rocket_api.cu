@@ -280,7 +280,7 @@ int rocket_params_set_path(rocket_params_t* p, int path) {
 int rocket_params_set_profiling(rocket_params_t* p, int enable) {
     if (!p || enable < 0 || enable > 1) return ROCKET_EINVAL;
     p->fast->profile = enable != 0;
-    if (!enable) p->fast->ev_valid = false;
+    if (!enable) p->fast->ev_chunks = 0;
     return ROCKET_OK;
 }
 
@@ -291,16 +291,23 @@ int rocket_params_last_profile(const rocket_params_t* p, double* ms_small_dilati
     if (flops_large_dilations) *flops_large_dilations = p->fast->host.flops_t;
     if (ms_small_dilations) *ms_small_dilations = 0.0;
     if (ms_large_dilations) *ms_large_dilations = 0.0;
-    if (!p->fast->ev_valid || p->device < 0) return ROCKET_OK;
+    if (p->fast->ev_chunks == 0 || p->device < 0) return ROCKET_OK;
     DeviceGuard g(p->device);
     if (!g.ok) return ROCKET_ECUDA;
-    cudaError_t e = cudaEventSynchronize(p->fast->ev[2]);
+    const std::vector<cudaEvent_t>& evs = p->fast->evs;
+    const int chunks = p->fast->ev_chunks;
+    cudaError_t e = cudaEventSynchronize(evs[3 * chunks - 1]);
     if (e != cudaSuccess) return cuda_status(e);
-    float a = 0.0f, b = 0.0f;
-    if ((e = cudaEventElapsedTime(&a, p->fast->ev[0], p->fast->ev[1])) != cudaSuccess) return cuda_status(e);
-    if ((e = cudaEventElapsedTime(&b, p->fast->ev[1], p->fast->ev[2])) != cudaSuccess) return cuda_status(e);
-    if (ms_small_dilations) *ms_small_dilations = a;
-    if (ms_large_dilations) *ms_large_dilations = b;
+    double ms_s = 0.0, ms_t = 0.0;
+    for (int c = 0; c < chunks; ++c) {
+        float a = 0.0f, b = 0.0f;
+        if ((e = cudaEventElapsedTime(&a, evs[3 * c], evs[3 * c + 1])) != cudaSuccess) return cuda_status(e);
+        if ((e = cudaEventElapsedTime(&b, evs[3 * c + 1], evs[3 * c + 2])) != cudaSuccess) return cuda_status(e);
+        ms_s += a;
+        ms_t += b;
+    }
+    if (ms_small_dilations) *ms_small_dilations = ms_s;
+    if (ms_large_dilations) *ms_large_dilations = ms_t;
     return ROCKET_OK;
 }
 

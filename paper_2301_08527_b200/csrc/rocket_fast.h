@@ -90,6 +90,7 @@ ROCKET_CX int t_stage_floats(int rg, int cg, int len) { return 4 * t_phase_float
 ROCKET_CX int imax_cx(int a, int b) { return a > b ? a : b; }
 constexpr int kTStageFloats = imax_cx(imax_cx(t_stage_floats(8, 1, ROCKET_MAX_LENGTH), t_stage_floats(4, 2, ROCKET_MAX_LENGTH)),
                                       t_stage_floats(2, 4, ROCKET_MAX_LENGTH));
+constexpr int kChunkExamples = 8;                                 // examples per pass through the fused kernels
 constexpr int kTPadFront = 128;                                    // zero floats before every channel row
 constexpr int kTXExtra = 256;                                      // floats a box may run past a 4d run
 
@@ -153,8 +154,8 @@ struct FastState {
     size_t soft_ws_bytes = 0;
     void* bwd_ws = nullptr;               // backward: fixed-point sums [n_weights + K], scales [K], max |x|
     bool profile = false;                 // record events around the S and T launches
-    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
-    bool ev_valid = false;
+    std::vector<cudaEvent_t> evs;         // three per chunk: before S, between S and T, after T
+    int ev_chunks = 0;                    // chunks of the last profiled call
 };
 
 // Uploads the plan (once per handle, at binding).

@@ -968,11 +968,9 @@ void release_fast_state(FastState& fs) {
     fs.bwd_ws = nullptr;
     fs.soft_ws = nullptr;
     fs.soft_ws_bytes = 0;
-    for (auto& ev : fs.ev) {
-        if (ev) cudaEventDestroy(ev);
-        ev = nullptr;
-    }
-    fs.ev_valid = false;
+    for (cudaEvent_t ev : fs.evs) cudaEventDestroy(ev);
+    fs.evs.clear();
+    fs.ev_chunks = 0;
     fs.plan_blob = fs.maps_blob = nullptr;
     fs.xpad = nullptr;
     fs.pad_examples = 0;
@@ -1032,7 +1030,7 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
     const size_t s_bytes = s_smem_bytes(dp.C), t_bytes = t_smem_bytes();
     const PlanDevice& pd = fs.dev;
     if (pd.n_titems > 0) {
-        e = ensure_pad_capacity(fs, N, dp.C, dp.L);
+        e = ensure_pad_capacity(fs, std::min(N, kChunkExamples), dp.C, dp.L);
         if (e != cudaSuccess) return e;
     }
     const int64_t pairs = (int64_t)N * dp.K;
@@ -1045,46 +1043,63 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
         fs.soft_ws_bytes = (size_t)pairs * 16;
     }
     FwdArgs a;
-    a.plan = fs.dev; a.X = X; a.feat_i = reinterpret_cast<int*>(feat);
-    a.ws = static_cast<unsigned long long*>(fs.soft_ws);
+    a.plan = fs.dev;
     a.c1 = lambda * 1.4426950408889634f; a.c0 = -shift * 1.4426950408889634f;
-    a.N = N; a.C = dp.C; a.L = dp.L; a.K = dp.K;
+    a.C = dp.C; a.L = dp.L; a.K = dp.K;
     a.dfeat = nullptr; a.argmax = nullptr; a.accfix = nullptr; a.scale = nullptr; a.n_weights = 0; a.lambda = lambda;
-    if (soft) fast_init_soft_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, stream>>>(a.ws, pairs, pd.counters);
-    else fast_init_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, stream>>>(a.feat_i, pairs, pd.counters);
+    int* feat_i = reinterpret_cast<int*>(feat);
+    unsigned long long* ws = static_cast<unsigned long long*>(fs.soft_ws);
+    if (soft) fast_init_soft_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, stream>>>(ws, pairs, pd.counters);
+    else fast_init_kernel<<<(unsigned)((pairs + 255) / 256), 256, 0, stream>>>(feat_i, pairs, pd.counters);
     count_launch();
-    if (pd.n_titems > 0) {
-        const int64_t rows = (int64_t)N * dp.C;
-        fast_pad_copy_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(X),
-                                                          fs.xpad, rows, dp.L / 4, fs.host.pad_pitch, kTPadFront,
-                                                          fs.copy_floats);
-        count_launch();
-    }
+    // the batch goes through in chunks of a few examples: the shifted copies of a chunk are read while
+    // they are still in L2, and they stay small
+    const int n_chunks = (N + kChunkExamples - 1) / kChunkExamples;
     if (fs.profile) {
-        for (auto& ev : fs.ev)
-            if (!ev && (e = cudaEventCreate(&ev)) != cudaSuccess) return e;
-        cudaEventRecord(fs.ev[0], stream);
+        while ((int)fs.evs.size() < 3 * n_chunks) {
+            cudaEvent_t ev = nullptr;
+            if ((e = cudaEventCreate(&ev)) != cudaSuccess) return e;
+            fs.evs.push_back(ev);
+        }
+        fs.ev_chunks = 0;
     }
-    if (pd.n_sitems > 0) {
-        const unsigned long long total = (unsigned long long)N * pd.n_sitems;
-        const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms);
-        if (soft) fast_s_forward<1><<<grid, kSThreads, s_bytes, stream>>>(a);
-        else fast_s_forward<0><<<grid, kSThreads, s_bytes, stream>>>(a);
-        count_launch();
-    }
-    if (fs.profile) cudaEventRecord(fs.ev[1], stream);
-    if (pd.n_titems > 0) {
-        if (soft) fast_t_forward<1><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
-        else fast_t_forward<0><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
-        count_launch();
-    }
-    if (fs.profile) {
-        cudaEventRecord(fs.ev[2], stream);
-        fs.ev_valid = true;
+    for (int c = 0; c < n_chunks; ++c) {
+        const int n0 = c * kChunkExamples, nc = std::min(kChunkExamples, N - n0);
+        a.X = X + (size_t)n0 * dp.C * dp.L;
+        a.feat_i = feat_i + (size_t)n0 * 2 * dp.K;
+        a.ws = ws ? ws + (size_t)n0 * 2 * dp.K : nullptr;
+        a.N = nc;
+        if (c > 0) {
+            e = cudaMemsetAsync(pd.counters, 0, 8, stream);
+            if (e != cudaSuccess) return e;
+        }
+        if (pd.n_titems > 0) {
+            fast_pad_copy_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(a.X), fs.xpad, (int64_t)nc * dp.C,
+                                                              dp.L / 4, fs.host.pad_pitch, kTPadFront, fs.copy_floats);
+            count_launch();
+        }
+        if (fs.profile) cudaEventRecord(fs.evs[3 * c], stream);
+        if (pd.n_sitems > 0) {
+            const unsigned long long total = (unsigned long long)nc * pd.n_sitems;
+            const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms);
+            if (soft) fast_s_forward<1><<<grid, kSThreads, s_bytes, stream>>>(a);
+            else fast_s_forward<0><<<grid, kSThreads, s_bytes, stream>>>(a);
+            count_launch();
+        }
+        if (fs.profile) cudaEventRecord(fs.evs[3 * c + 1], stream);
+        if (pd.n_titems > 0) {
+            if (soft) fast_t_forward<1><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
+            else fast_t_forward<0><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
+            count_launch();
+        }
+        if (fs.profile) {
+            cudaEventRecord(fs.evs[3 * c + 2], stream);
+            fs.ev_chunks = c + 1;
+        }
     }
     const int64_t fin = (int64_t)N * pd.n_krec;
     if (fin > 0) {
-        if (soft) fast_finalize_soft_kernel<<<(unsigned)((fin + 255) / 256), 256, 0, stream>>>(feat, argmax, a.ws, pd.krec, pd.n_krec, N, dp.K);
+        if (soft) fast_finalize_soft_kernel<<<(unsigned)((fin + 255) / 256), 256, 0, stream>>>(feat, argmax, ws, pd.krec, pd.n_krec, N, dp.K);
         else fast_finalize_kernel<<<(unsigned)((fin + 255) / 256), 256, 0, stream>>>(feat, pd.krec, pd.n_krec, N, dp.K);
         count_launch();
     }
@@ -1113,7 +1128,7 @@ cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t 
     double* scale = reinterpret_cast<double*>(static_cast<char*>(fs.bwd_ws) + acc_bytes);
     unsigned* absmax = reinterpret_cast<unsigned*>(static_cast<char*>(fs.bwd_ws) + acc_bytes + scale_bytes);
     if (pd.n_titems > 0 && N > 0) {
-        e = ensure_pad_capacity(fs, N, dp.C, dp.L);
+        e = ensure_pad_capacity(fs, std::min(N, kChunkExamples), dp.C, dp.L);
         if (e != cudaSuccess) return e;
     }
     e = cudaMemsetAsync(absmax, 0, 256, stream);
@@ -1127,22 +1142,25 @@ cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t 
                                                                          accfix, n_weights);
     count_launch();
     FwdArgs a;
-    a.plan = fs.dev; a.X = X; a.feat_i = nullptr; a.ws = nullptr;
+    a.plan = fs.dev; a.feat_i = nullptr; a.ws = nullptr;
     a.c1 = lambda * 1.4426950408889634f; a.c0 = -shift * 1.4426950408889634f;
-    a.N = N; a.C = dp.C; a.L = dp.L; a.K = dp.K;
-    a.dfeat = dfeat; a.argmax = argmax; a.accfix = accfix; a.scale = scale; a.n_weights = n_weights; a.lambda = lambda;
-    if (N > 0) {
-        fast_init_kernel<<<1, 32, 0, stream>>>(nullptr, 0, pd.counters);  // resets the S work counter
-        count_launch();
+    a.C = dp.C; a.L = dp.L; a.K = dp.K;
+    a.accfix = accfix; a.scale = scale; a.n_weights = n_weights; a.lambda = lambda;
+    for (int n0 = 0; n0 < N; n0 += kChunkExamples) {
+        const int nc = std::min(kChunkExamples, N - n0);
+        a.X = X + (size_t)n0 * dp.C * dp.L;
+        a.dfeat = dfeat + (size_t)n0 * 2 * dp.K;
+        a.argmax = argmax + (size_t)n0 * dp.K;
+        a.N = nc;
+        e = cudaMemsetAsync(pd.counters, 0, 8, stream);
+        if (e != cudaSuccess) return e;
         if (pd.n_titems > 0) {
-            const int64_t rows = (int64_t)N * dp.C;
-            fast_pad_copy_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(X),
-                                                              fs.xpad, rows, dp.L / 4, fs.host.pad_pitch,
-                                                              kTPadFront, fs.copy_floats);
+            fast_pad_copy_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(a.X), fs.xpad, (int64_t)nc * dp.C,
+                                                              dp.L / 4, fs.host.pad_pitch, kTPadFront, fs.copy_floats);
             count_launch();
         }
         if (pd.n_sitems > 0) {
-            const unsigned long long total = (unsigned long long)N * pd.n_sitems;
+            const unsigned long long total = (unsigned long long)nc * pd.n_sitems;
             const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms);
             fast_s_forward<2><<<grid, kSThreads, s_bytes, stream>>>(a);
             count_launch();
