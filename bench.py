@@ -35,7 +35,7 @@ LAMBDA, SHIFT = 10.0, 3.0
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the committed ncu capture
 # (profiles/); None until a capture of the current kernel exists.
-NCU_DRAM_BYTES_PER_LAUNCH = {"fast_s_forward": 38.3e6 * 60 / 8, "fast_t_forward": 64.1e6 * 60 / 8}
+NCU_DRAM_BYTES_PER_LAUNCH = {"fast_s_forward": 38.3e6, "fast_t_forward": 827.5e6}   # per launch = one chunk of 8 examples
 
 
 def fp32_peak_tflops(sm_count, sm_mhz):
@@ -281,7 +281,8 @@ def main():
     peak = fp32_peak_tflops(props.multi_processor_count, sm_max)
     roofline = {"bound": "alu", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(dom.split()[0]),
-                "launch_ms": dom_ms,
+                "launch_ms": dom_ms, "launches_per_step": (w["N"] + 7) // 8,
+                "traffic_note": "ncu, cold cache, one launch = one chunk of 8 examples (32 MB of input)",
                 "peak_source": "derived: %d SMs x 128 FP32 lanes x 2 flop x %.0f MHz (max SM clock from %s); "
                                "a packed-FMA microbenchmark reaches 74.0 TFLOP/s on this pool" % (
                                    props.multi_processor_count, sm_max,

@@ -178,8 +178,9 @@ int rocket_params_device_status(const rocket_params_t* p, int* wait_timeouts);
  * rocket_transform call through the fast path records CUDA events on the caller's stream around
  * its two fused kernels: the one that serves the small dilations (tiles shared by all kernels of
  * one dilation) and the one that serves the large dilations (one kernel per tile).
- * rocket_params_last_profile waits for the last such call and returns the two durations in
- * milliseconds (0 when nothing was recorded), and the convolution work of one example in either
+ * The batch goes through both kernels in chunks of a few examples; rocket_params_last_profile waits
+ * for the last such call and returns the two durations, summed over the chunks, in milliseconds
+ * (0 when nothing was recorded), and the convolution work of one example in either
  * kernel under the count 2*len*channels*L_out (flop).  Any output pointer may be NULL.
  */
 int rocket_params_set_profiling(rocket_params_t* p, int enable);
