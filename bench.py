@@ -100,6 +100,22 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(value, world, device="cuda"):
+    """Max of a python float over the ranks of the default process group (identity for one rank)."""
+    if world == 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(examples_per_rank, steps, seconds_max_over_ranks, world):
+    """Whole-job throughput: every rank transforms its own batch (weak scaling), the slowest rank sets the time."""
+    return world * examples_per_rank * steps / seconds_max_over_ranks
+
+
 def run_reference(args, rank):
     """The CPU oracle, as it stands, on the machine's host cores: a bounded sample of the workload per step."""
     if rank != 0:
@@ -196,12 +212,8 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(v):
-        if world == 1:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    def max_over(v):
+        return max_over_ranks(v, world)
 
     w = dict(WORKLOAD)
     if args.small:
@@ -246,9 +258,9 @@ def main():
     clocks = sampler.stop() if sampler else None
     launches = rk.kernel_launch_count() - launches0
     launches_timed = launches * args.steps // (args.steps + args.warmup)
-    total_s = max_over_ranks(total_s)
+    total_s = max_over(total_s)
     ms_per_step = 1e3 * total_s / args.steps
-    value = world * w["N"] * args.steps / total_s
+    value = whole_job_value(w["N"], args.steps, total_s, world)
 
     # end to end through the host-buffer entry point: H2D of X and D2H of the features inside the timing
     def e2e_step():
@@ -261,7 +273,7 @@ def main():
     for _ in range(e2e_steps):
         e2e_step()
     barrier()
-    e2e_s = max_over_ranks(time.perf_counter() - t0)
+    e2e_s = max_over(time.perf_counter() - t0)
     e2e = {"value": world * w["N"] * e2e_steps / e2e_s, "unit": UNIT,
            "h2d_bytes_per_step": X_host.numel() * 4, "d2h_bytes_per_step": feat_host.numel() * 4,
            "steps": e2e_steps, "api": "rocket_transform_host (pinned host buffers)"}
@@ -310,7 +322,7 @@ def main():
                                psteps, 3)
         s_bwd, _ = time_steps(lambda: rk.rocket_transform_soft_backward(params, Xt, LAMBDA, SHIFT, g, arg, dW, db),
                               psteps, 3)
-        s_soft, s_bwd = max_over_ranks(s_soft) / psteps, max_over_ranks(s_bwd) / psteps
+        s_soft, s_bwd = max_over(s_soft) / psteps, max_over(s_bwd) / psteps
         passes = {
             "shape": "N=32 x C=20 x L=50000, K=10000 (config 3), lambda=%g, shift=%g" % (LAMBDA, SHIFT),
             "soft_forward": {"examples_per_s": world * t["N"] / s_soft, "ms": 1e3 * s_soft,
