@@ -17,8 +17,9 @@
 //     channels in shared memory, then its warps pull kernels of the bucket from a shared
 //     counter, so one staged tile serves dozens to hundreds of kernels.
 //   T (d >= split): few kernels share a dilation, so a block of eight consumer warps takes one
-//     kernel and one tile of up to eight warp tiles (128 x 64, 64 x 128 or 32 x 256) and streams the
-//     kernel's channels through a ring of shared-memory stages.  A producer warp fills the
+//     kernel and one tile of up to eight warp tiles (128 x 64, 64 x 128, 32 x 256, or 16 x 512 for
+//     kernels whose outputs span at most 16 rows of A) and streams the kernel's channels through a
+//     ring of shared-memory stages.  A producer warp fills the
 //     ring with tiled TMA loads from a zero-margined copy of the batch, viewed as a 3-D tensor
 //     (x within a run of 4d floats, y = which run, z = channel row): rows s, s+4, s+8, .. of
 //     a tile are then one box, and four boxes (one per s mod 4) bring a whole stage without
@@ -90,6 +91,7 @@ ROCKET_CX int t_stage_floats(int rg, int cg, int len) { return 4 * t_phase_float
 ROCKET_CX int imax_cx(int a, int b) { return a > b ? a : b; }
 constexpr int kTStageFloats = imax_cx(imax_cx(t_stage_floats(8, 1, ROCKET_MAX_LENGTH), t_stage_floats(4, 2, ROCKET_MAX_LENGTH)),
                                       t_stage_floats(2, 4, ROCKET_MAX_LENGTH));
+constexpr int kTWideCols = 256;                                    // columns of one half of a wide tile
 constexpr int kChunkExamples = 8;                                 // examples per pass through the fused kernels
 constexpr int kTPadFront = 128;                                    // zero floats before every channel row
 constexpr int kTXExtra = 256;                                      // floats a box may run past a 4d run
@@ -100,8 +102,9 @@ struct alignas(16) TItem {
     int32_t d, len, m, box_rows;
     uint8_t ch[12];
     int32_t krec;                         // index into the kernel records
-    int32_t cg, pad0_[3];
-    int32_t x[4], y[4];                   // tensor coordinates of the four phase boxes
+    int32_t cg, wide, g_lo, g_hi;         // wide tile: 1 x 8 warp tiles as two halves of 256 columns, of which only
+                                          // the groups of four rows [g_lo, g_hi) are loaded (box_rows = g_hi - g_lo)
+    int32_t x[4], y[4];                   // tensor coordinates of the four phase boxes (first half; y of group g_lo)
     int32_t j[4];                         // which shifted copy each phase reads
     int32_t pad1_[4];
 };

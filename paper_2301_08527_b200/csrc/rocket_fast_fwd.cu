@@ -60,10 +60,12 @@ __device__ __forceinline__ float key_float(int k) { return __int_as_float(k >= 0
 
 // One channel of one warp tile: 16 output rows of the thread's column pair, 16+ELL-1 input pairs
 // streamed past them.  Row s of the tile sits at st[off[s & 3] + (s >> 2) * STEP]; w2 holds the
-// channel's negated weights, each twice.
-template <int ELL, int STEP>
+// channel's negated weights, each twice.  With WIN, only the groups of four rows [gl, gh) are read
+// and multiplied (the others hold no sample and are not in shared memory); gl and gh are the same
+// for the whole warp.
+template <int ELL, int STEP, bool WIN>
 __device__ __forceinline__ void conv_channel(const float* __restrict__ st, const int (&off)[4],
-                                             const float* __restrict__ w2, u64 (&acc)[kR]) {
+                                             const float* __restrict__ w2, u64 (&acc)[kR], int gl = 0, int gh = 0) {
     u64 wp[ELL + 1];
 #pragma unroll
     for (int j = 0; j < ELL; j += 2) {
@@ -72,13 +74,18 @@ __device__ __forceinline__ void conv_channel(const float* __restrict__ st, const
         wp[j + 1] = v.y;
     }
 #pragma unroll
-    for (int s = 0; s < kR + ELL - 1; ++s) {
-        const float* p = st + off[s & 3] + (s >> 2) * STEP;
-        const u64 x = *reinterpret_cast<const u64*>(p);
+    for (int g = 0; g < (kR + ELL - 1 + 3) / 4; ++g) {
+        if (!WIN || (g >= gl && g < gh)) {
 #pragma unroll
-        for (int j = 0; j < ELL; ++j) {
-            const int o = s - j;
-            if (o >= 0 && o < kR) fma2(acc[o], wp[j], x);
+            for (int s = 4 * g; s < 4 * g + 4 && s < kR + ELL - 1; ++s) {
+                const float* p = st + off[s & 3] + (s >> 2) * STEP;
+                const u64 x = *reinterpret_cast<const u64*>(p);
+#pragma unroll
+                for (int j = 0; j < ELL; ++j) {
+                    const int o = s - j;
+                    if (o >= 0 && o < kR) fma2(acc[o], wp[j], x);
+                }
+            }
         }
     }
 }
@@ -240,17 +247,22 @@ __device__ __forceinline__ float make_gz(u64 (&acc)[kR], float c1, float c0, flo
 
 // Backward, second half, one channel of one warp tile: dw[j] += gz[o] * x[o + j] for the thread's
 // column pair (same traversal as conv_channel with the roles of weights and accumulators swapped).
-template <int ELL, int STEP>
+template <int ELL, int STEP, bool WIN>
 __device__ __forceinline__ void grad_channel(const float* __restrict__ st, const int (&off)[4], const u64 (&gz)[kR],
-                                             u64 (&dw)[ELL]) {
+                                             u64 (&dw)[ELL], int gl = 0, int gh = 0) {
 #pragma unroll
-    for (int s = 0; s < kR + ELL - 1; ++s) {
-        const float* p = st + off[s & 3] + (s >> 2) * STEP;
-        const u64 x = *reinterpret_cast<const u64*>(p);
+    for (int g = 0; g < (kR + ELL - 1 + 3) / 4; ++g) {
+        if (!WIN || (g >= gl && g < gh)) {
 #pragma unroll
-        for (int j = 0; j < ELL; ++j) {
-            const int o = s - j;
-            if (o >= 0 && o < kR) fma2(dw[j], gz[o], x);
+            for (int s = 4 * g; s < 4 * g + 4 && s < kR + ELL - 1; ++s) {
+                const float* p = st + off[s & 3] + (s >> 2) * STEP;
+                const u64 x = *reinterpret_cast<const u64*>(p);
+#pragma unroll
+                for (int j = 0; j < ELL; ++j) {
+                    const int o = s - j;
+                    if (o >= 0 && o < kR) fma2(dw[j], gz[o], x);
+                }
+            }
         }
     }
 }
@@ -332,7 +344,7 @@ __device__ __forceinline__ void s_grad_tile(const float* planes, const KRec* rec
         u64 dw[ELL];
 #pragma unroll
         for (int j = 0; j < ELL; ++j) dw[j] = 0ull;
-        grad_channel<ELL, 4 * kWarpCols>(planes + rec->ch[q] * kSPlaneFloats, off, gz, dw);
+        grad_channel<ELL, 4 * kWarpCols, false>(planes + rec->ch[q] * kSPlaneFloats, off, gz, dw);
         reduce_publish_dw<ELL>(dw, accfix + rec->woff + q * ELL, scale, lane);
     }
 }
@@ -342,7 +354,7 @@ __device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* r
     const int m = rec->m;
     const int off[4] = {2 * lane, kWarpCols + 2 * lane, 2 * kWarpCols + 2 * lane, 3 * kWarpCols + 2 * lane};
     for (int q = 0; q < m; ++q)
-        conv_channel<ELL, 4 * kWarpCols>(planes + rec->ch[q] * kSPlaneFloats, off, rec->w2[q], acc);
+        conv_channel<ELL, 4 * kWarpCols, false>(planes + rec->ch[q] * kSPlaneFloats, off, rec->w2[q], acc);
 }
 
 template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft
@@ -512,7 +524,8 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, int 
 // What the producer tells the consumers about a tile (written with plain stores before its
 // arrive on the stage's barrier, which releases them).
 struct TSlotItem {
-    int32_t t0, r0, rg, cg, box_rows, rec_slot, pad_[2];
+    int32_t t0, r0, rg, cg, box_rows, rec_slot, wide, g_lo;
+    int32_t g_hi, pad_[3];
 };
 
 struct TShared {
@@ -524,14 +537,15 @@ struct TShared {
 
 // The channels of one tile for one consumer warp; returns false when a wait gave up.  A warp
 // without a valid output (active == false) only keeps the ring moving.
-template <int ELL, int STEP>
+template <int ELL, int STEP, bool WIN>
 __device__ __forceinline__ bool t_channels(const float* stages, const KRec* rec, const int (&off)[4], uint32_t full0,
-                                           uint32_t empty0, uint32_t& st, int lane, bool active, u64 (&acc)[kR]) {
+                                           uint32_t empty0, uint32_t& st, int lane, bool active, u64 (&acc)[kR], int gl,
+                                           int gh) {
     const int m = rec->m;
     for (int q = 0; q < m; ++q) {
         const uint32_t slot = st % kTStages;
         if (q > 0 && !mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) return false;
-        if (active) conv_channel<ELL, STEP>(stages + slot * kTStageFloats, off, rec->w2[q], acc);
+        if (active) conv_channel<ELL, STEP, WIN>(stages + slot * kTStageFloats, off, rec->w2[q], acc, gl, gh);
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * slot);
         ++st;
@@ -540,10 +554,10 @@ __device__ __forceinline__ bool t_channels(const float* stages, const KRec* rec,
 }
 
 // Backward second half on a T tile: the kernel's channels stream through the ring once more.
-template <int ELL, int STEP>
+template <int ELL, int STEP, bool WIN>
 __device__ __forceinline__ bool t_grad_channels(const float* stages, const KRec* rec, const int (&off)[4], uint32_t full0,
                                                 uint32_t empty0, uint32_t& st, int lane, bool active, const u64 (&gz)[kR],
-                                                long long* accfix, double scale) {
+                                                long long* accfix, double scale, int gl, int gh) {
     const int m = rec->m;
     for (int q = 0; q < m; ++q) {
         const uint32_t slot = st % kTStages;
@@ -552,7 +566,7 @@ __device__ __forceinline__ bool t_grad_channels(const float* stages, const KRec*
             u64 dw[ELL];
 #pragma unroll
             for (int j = 0; j < ELL; ++j) dw[j] = 0ull;
-            grad_channel<ELL, STEP>(stages + slot * kTStageFloats, off, gz, dw);
+            grad_channel<ELL, STEP, WIN>(stages + slot * kTStageFloats, off, gz, dw, gl, gh);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + 8u * slot);
             reduce_publish_dw<ELL>(dw, accfix + rec->woff + q * ELL, scale, lane);
@@ -565,22 +579,22 @@ __device__ __forceinline__ bool t_grad_channels(const float* stages, const KRec*
     return true;
 }
 
-template <int STEP>
+template <int STEP, bool WIN>
 __device__ __forceinline__ bool t_grad_dispatch(int len, const float* stages, const KRec* rec, const int (&off)[4],
                                                 uint32_t full0, uint32_t empty0, uint32_t& st, int lane, bool active,
-                                                const u64 (&gz)[kR], long long* accfix, double scale) {
-    if (len == 7) return t_grad_channels<7, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale);
-    if (len == 9) return t_grad_channels<9, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale);
-    return t_grad_channels<11, STEP>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale);
+                                                const u64 (&gz)[kR], long long* accfix, double scale, int gl, int gh) {
+    if (len == 7) return t_grad_channels<7, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale, gl, gh);
+    if (len == 9) return t_grad_channels<9, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale, gl, gh);
+    return t_grad_channels<11, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, gz, accfix, scale, gl, gh);
 }
 
-template <int STEP>
+template <int STEP, bool WIN>
 __device__ __forceinline__ bool t_dispatch(int len, const float* stages, const KRec* rec, const int (&off)[4],
                                            uint32_t full0, uint32_t empty0, uint32_t& st, int lane, bool active,
-                                           u64 (&acc)[kR]) {
-    if (len == 7) return t_channels<7, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
-    if (len == 9) return t_channels<9, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
-    return t_channels<11, STEP>(stages, rec, off, full0, empty0, st, lane, active, acc);
+                                           u64 (&acc)[kR], int gl, int gh) {
+    if (len == 7) return t_channels<7, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
+    if (len == 9) return t_channels<9, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
+    return t_channels<11, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
 }
 
 template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft
@@ -620,9 +634,10 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                 for (int i = i_beg; ok && i < i_end; ++i) {
                     if (*abort_flag) { ok = false; break; }
                     const int map = w0.x, t0 = w0.y, r0 = w0.z, rg = w0.w;
-                    const int m = w1.z, box_rows = w1.w, krec = w2.w, cg = w3.x;
+                    const int m = w1.z, box_rows = w1.w, krec = w2.w, cg = w3.x, wide = w3.y, g_lo = w3.z, g_hi = w3.w;
                     const unsigned chw[3] = {(unsigned)w2.x, (unsigned)w2.y, (unsigned)w2.z};
                     const int px[4] = {w4.x, w4.y, w4.z, w4.w}, py[4] = {w5.x, w5.y, w5.z, w5.w}, pj[4] = {w6.x, w6.y, w6.z, w6.w};
+                    const int run = 4 * w1.x;
                     {   // the next tile's description is on its way while this one is issued
                         int inext = i + 1;
                         if (inext == i_end) inext = i_beg;
@@ -645,10 +660,11 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                             break;
                         }
                         const uint32_t bar = full0 + 8u * slot;
-                        uint32_t tx = 4u * box_bytes;
+                        uint32_t tx = (wide ? 8u : 4u) * box_bytes;
                         if (q2 == 0) {
                             TSlotItem& si = sh.items[it % kTParamSlots];
                             si.t0 = t0; si.r0 = r0; si.rg = rg; si.cg = cg; si.box_rows = box_rows; si.rec_slot = (int)rslot;
+                            si.wide = wide; si.g_lo = g_lo; si.g_hi = g_hi;
                             if (new_rec) tx += (uint32_t)sizeof(KRec);
                         }
                         mbar_arrive_expect_tx(bar, tx);
@@ -658,6 +674,14 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                         const uint32_t dst0 = smem_u32(stages + slot * kTStageFloats);
 #pragma unroll
                         for (int k = 0; k < 4; ++k) tma_load_4d(dst0 + (uint32_t)k * phase_bytes, tmap, px[k], py[k], z, pj[k], bar);
+                        if (wide) {   // the second half: the boxes 256 columns further right
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                int x2 = px[k] + kTWideCols, y2 = py[k];
+                                if (x2 >= run) { x2 -= run; ++y2; }
+                                tma_load_4d(dst0 + (uint32_t)(4 + k) * phase_bytes, tmap, x2, y2, z, pj[k], bar);
+                            }
+                        }
                         ++st;
                     }
                     ++it;
@@ -690,7 +714,10 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                 const KRec* rec = recs + si.rec_slot;
                 const int t0 = si.t0, r0 = si.r0, rg = si.rg, cg = si.cg, box_rows = si.box_rows;
                 const int len = rec->len, d = rec->d, korig = rec->k;
-                const int wr = cg == 1 ? warp : (cg == 2 ? warp >> 1 : warp >> 2), wc = warp & (cg - 1);
+                const bool wide = si.wide != 0;
+                // warp tile (wr, wc) of the tile; a wide tile is one row of eight
+                const int wr = wide ? 0 : (cg == 1 ? warp : (cg == 2 ? warp >> 1 : warp >> 2));
+                const int wc = wide ? warp : (warp & (cg - 1));
                 const int lc = kWarpCols * wc + 2 * lane;
                 const bool in_tile = wr < rg;
                 const bool ok0 = in_tile && r0 + lc < d, ok1 = in_tile && r0 + lc + 1 < d;
@@ -702,12 +729,16 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                 const int boxw = t_box_cols(cg);
                 int off[4];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) off[k] = t_box_offset(cg, k, box_rows) + 4 * wr * boxw + lc;
+                for (int k = 0; k < 4; ++k)
+                    off[k] = wide ? t_wide_elem_offset(k, lc, box_rows, si.g_lo)
+                                  : t_box_offset(cg, k, box_rows) + 4 * wr * boxw + lc;
+                const int gl = si.g_lo, gh = si.g_hi;
                 u64 acc[kR];
                 init_acc(acc, rec->negb, interior, lo0, hi0, lo1, hi1);
-                if (cg == 1) ok = t_dispatch<kWarpCols>(len, stages, rec, off, full0, empty0, st, lane, active, acc);
-                else if (cg == 2) ok = t_dispatch<2 * kWarpCols>(len, stages, rec, off, full0, empty0, st, lane, active, acc);
-                else ok = t_dispatch<4 * kWarpCols>(len, stages, rec, off, full0, empty0, st, lane, active, acc);
+                if (wide) ok = t_dispatch<kTWideCols, true>(len, stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
+                else if (cg == 1) ok = t_dispatch<kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
+                else if (cg == 2) ok = t_dispatch<2 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
+                else ok = t_dispatch<4 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
                 if (!ok) break;
                 if (MODE == 2) {
                     const int64_t pair = (int64_t)n * a.K + korig;
@@ -727,9 +758,10 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                         scale = __ldg(a.scale + korig);
                         if (lane == 0) add_fixed(a.accfix + a.n_weights + korig, dbs, scale);
                     }
-                    if (cg == 1) ok = t_grad_dispatch<kWarpCols>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale);
-                    else if (cg == 2) ok = t_grad_dispatch<2 * kWarpCols>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale);
-                    else ok = t_grad_dispatch<4 * kWarpCols>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale);
+                    if (wide) ok = t_grad_dispatch<kTWideCols, true>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale, gl, gh);
+                    else if (cg == 1) ok = t_grad_dispatch<kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale, 0, 0);
+                    else if (cg == 2) ok = t_grad_dispatch<2 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale, 0, 0);
+                    else ok = t_grad_dispatch<4 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale, 0, 0);
                     if (!ok) break;
                 } else if (active) {
                     if (MODE == 1) {

@@ -60,12 +60,44 @@ ROCKET_HD TPhase t_phase(int t0, int r0, int d, int k) {
     return p;
 }
 
+// The box `cols` floats to the right of box p in the same row of A (same shifted copy when cols
+// is a multiple of 4).
+ROCKET_HD TPhase t_phase_right(TPhase p, int cols, int d) {
+    p.x += cols;
+    if (p.x >= 4 * d) { p.x -= 4 * d; p.y += 1; }
+    return p;
+}
+
+// Rows of A that hold samples are [0, ceil(L / d)): every other row is zero.  A wide tile loads
+// and multiplies only the groups of four tile rows [g_lo, g_hi) that hold samples (at least one
+// group, so that a box is never empty).
+struct TWindow { int g_lo, g_hi; };
+
+ROCKET_HD TWindow t_window(int t0, int rows, int d, int L) {
+    const int t_data = (L + d - 1) / d;
+    const int s_lo = -t0 > 0 ? -t0 : 0;
+    const int s_hi = imin(rows, t_data - t0);
+    TWindow w;
+    if (s_hi <= s_lo) { w.g_lo = 0; w.g_hi = 1; return w; }
+    w.g_lo = s_lo >> 2;
+    w.g_hi = (s_hi + 3) >> 2;
+    return w;
+}
+
 // Float offset, inside a stage, of the box of phase k.
 ROCKET_HD int t_box_offset(int cg, int k, int box_rows) { return k * t_phase_floats(cg, box_rows); }
 
 // Float offset, inside a stage, of tile row s / tile column lc as the consumer reads it.
 ROCKET_HD int t_elem_offset(int cg, int s, int lc, int box_rows) {
     return t_box_offset(cg, s & 3, box_rows) + (s >> 2) * t_box_cols(cg) + lc;
+}
+
+// The same for a wide tile: column lc in [0, 512) lies in half lc / 256; row s must belong to a
+// loaded group (g_lo <= s / 4 < g_lo + box_rows).
+ROCKET_HD int t_wide_half_floats(int box_rows) { return 4 * t_phase_floats(4, box_rows); }
+ROCKET_HD int t_wide_elem_offset(int s, int lc, int box_rows, int g_lo) {
+    return (lc / kTWideCols) * t_wide_half_floats(box_rows) + t_box_offset(4, s & 3, box_rows) +
+           ((s >> 2) - g_lo) * kTWideCols + (lc % kTWideCols);
 }
 
 }  // namespace fast

@@ -118,6 +118,11 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
             if (rest >= 2) { widths.push_back(2); rest -= 2; }
             if (rest >= 1) widths.push_back(1);
         };
+        // kernels whose outputs span at most 16 rows of A: wide tiles (8 column groups side by side,
+        // only the rows that hold samples), as long as two halves fit a stage
+        const int t_first = (int)tmin;
+        const TWindow win = t_window(t_first, kR + f.len - 1, f.d, hp.L);
+        const bool wide_ok = R16 == 1 && 2 * t_wide_half_floats(win.g_hi - win.g_lo) <= kTStageFloats;
         int best_cg = 2;
         int64_t best_tiles = INT64_MAX;
         for (int cg : {2, 4, 1}) {
@@ -128,29 +133,52 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
             if (tiles < best_tiles) { best_tiles = tiles; best_cg = cg; }
         }
         std::vector<int> widths;
-        chunks_of(best_cg, widths);
+        if (wide_ok) {
+            widths.assign(C64 / 8, 8);
+            int rest = C64 % 8;
+            if (rest >= 5) { widths.push_back(8); rest = 0; }
+            if (rest >= 3) { widths.push_back(4); rest = rest > 4 ? rest - 4 : 0; }
+            if (rest >= 2) { widths.push_back(2); rest -= 2; }
+            if (rest >= 1) widths.push_back(1);
+        } else {
+            chunks_of(best_cg, widths);
+        }
         int c64 = 0;
         for (int w : widths) {
-            const int rg_full = 8 / w;
+            const int rg_full = w == 8 ? 1 : 8 / w;
             for (int r16 = 0; r16 < R16; r16 += rg_full) {
                 TItem it{};
-                it.rg = std::min(rg_full, R16 - r16); it.cg = w;
+                it.rg = std::min(rg_full, R16 - r16);
+                it.wide = w == 8 ? 1 : 0;
+                it.cg = it.wide ? 4 : w;
                 it.t0 = (int32_t)(tmin + (int64_t)kR * r16); it.r0 = c64 * kWarpCols;
-                it.d = f.d; it.len = f.len; it.m = f.m; it.box_rows = t_box_rows(it.rg, f.len);
+                // a tile none of whose (row, column) pairs is an output of the kernel is left out
+                bool any_output = false;
+                for (int t = it.t0; t < it.t0 + kR * it.rg && !any_output; ++t) {
+                    const int64_t c_lo = std::max<int64_t>(it.r0, (int64_t)f.lo_u - (int64_t)t * f.d);
+                    const int64_t c_hi = std::min<int64_t>(std::min(it.r0 + kWarpCols * w, f.d), (int64_t)f.hi_u - (int64_t)t * f.d);
+                    any_output = c_lo < c_hi;
+                }
+                if (!any_output) continue;
+                it.d = f.d; it.len = f.len; it.m = f.m;
+                it.g_lo = it.wide ? win.g_lo : 0;
+                it.g_hi = it.wide ? win.g_hi : t_box_rows(it.rg, f.len);
+                it.box_rows = it.g_hi - it.g_lo;
                 for (int q = 0; q < f.m; ++q) it.ch[q] = (uint8_t)f.ch[q];
                 it.krec = ki;
-                const auto key = std::make_tuple(f.d, t_box_cols(w), it.box_rows);
+                const auto key = std::make_tuple(f.d, t_box_cols(it.cg), it.box_rows);
                 auto found = map_index.find(key);
                 if (found == map_index.end()) {
                     found = map_index.emplace(key, (int)out.tmaps.size()).first;
-                    out.tmaps.push_back({f.d, t_box_cols(w), it.box_rows});
+                    out.tmaps.push_back({f.d, t_box_cols(it.cg), it.box_rows});
                 }
                 it.map = found->second;
                 for (int ph = 0; ph < 4; ++ph) {
                     const TPhase tp = t_phase(it.t0, it.r0, it.d, ph);
-                    it.x[ph] = tp.x; it.y[ph] = tp.y; it.j[ph] = tp.j;
+                    it.x[ph] = tp.x; it.y[ph] = tp.y + it.g_lo; it.j[ph] = tp.j;
                 }
-                out.tcost.push_back((double)f.m * (f.len + 2) + 8.0);
+                const double share = it.wide ? (double)it.box_rows / t_box_rows(1, f.len) : 1.0;
+                out.tcost.push_back((double)f.m * (f.len * share + 2) + 8.0);
                 out.titems.push_back(it);
             }
             c64 += w;

@@ -89,18 +89,34 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
         REQUIRE((it.cg == 1 || it.cg == 2 || it.cg == 4) && it.rg >= 1 && it.rg * it.cg <= kTConsumerWarps, "T shape");
         REQUIRE(it.r0 % kWarpCols == 0 && it.r0 < f.d, "T column origin");
         for (int q = 0; q < f.m; ++q) REQUIRE(it.ch[q] == f.ch[q], "T channel list");
-        const int rows_out = kR * it.rg, groups = it.cg, boxw = t_box_cols(it.cg);
+        const bool wide = it.wide != 0;
+        const int rows_out = kR * it.rg, boxw = t_box_cols(it.cg);
+        const int tile_cols = wide ? 2 * kTWideCols : boxw;
         const int rows = rows_out + f.len - 1;
-        REQUIRE(it.box_rows == t_box_rows(it.rg, f.len) && 4 * it.box_rows >= rows, "T box rows");
+        if (wide) {
+            const TWindow win = t_window(it.t0, rows, f.d, L);
+            REQUIRE(it.rg == 1 && it.cg == 4 && boxw == kTWideCols, "wide tile shape");
+            REQUIRE(it.g_lo == win.g_lo && it.g_hi == win.g_hi && win.g_lo >= 0 && win.g_lo < win.g_hi && 4 * win.g_hi < rows + 4,
+                    "wide tile window");
+            REQUIRE(2 * t_wide_half_floats(it.box_rows) <= kTStageFloats, "wide stage size");
+        } else {
+            REQUIRE(it.g_lo == 0 && it.g_hi == t_box_rows(it.rg, f.len) && 4 * it.g_hi >= rows, "T box rows");
+        }
+        REQUIRE(it.box_rows == it.g_hi - it.g_lo, "T box rows and window");
         REQUIRE(sp.d == f.d && sp.box_cols == boxw && sp.box_rows == it.box_rows && boxw <= 256 && it.box_rows <= 256, "T map spec");
         REQUIRE(4 * t_phase_floats(it.cg, it.box_rows) <= kTStageFloats, "stage size");
         const long long run = 4ll * f.d, ny = (kTPadFront + (long long)L + run - 1) / run;
-        // the boxes the producer issues
-        TPhase ph[4];
-        for (int k = 0; k < 4; ++k) {
-            ph[k] = t_phase(it.t0, it.r0, f.d, k);
+        // the boxes the producer issues: four phases, twice for a wide tile
+        TPhase ph[8];
+        for (int k = 0; k < (wide ? 8 : 4); ++k) {
+            if (k < 4) {
+                ph[k] = t_phase(it.t0, it.r0, f.d, k);
+                ph[k].y += it.g_lo;
+                REQUIRE(it.x[k] == ph[k].x && it.y[k] == ph[k].y && it.j[k] == ph[k].j, "stored box coordinates");
+            } else {
+                ph[k] = t_phase_right(ph[k - 4], kTWideCols, f.d);
+            }
             REQUIRE(ph[k].x % 4 == 0 && ph[k].x >= 0 && ph[k].x < run && ph[k].j >= 0 && ph[k].j < 4, "box x");
-            REQUIRE(it.x[k] == ph[k].x && it.y[k] == ph[k].y && it.j[k] == ph[k].j, "stored box coordinates");
             REQUIRE(ph[k].x + boxw <= run + kTXExtra, "box leaves the tensor row");
             const int dst = t_box_offset(it.cg, k, it.box_rows);
             REQUIRE(dst % 32 == 0 && dst + it.box_rows * boxw <= kTStageFloats, "box destination");
@@ -114,7 +130,7 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
             }
         }
         // what every consumer thread owns and reads
-        for (int lc = 0; lc < kWarpCols * groups; ++lc) {
+        for (int lc = 0; lc < tile_cols; ++lc) {
             const bool col_ok = it.r0 + lc < f.d;
             for (int wr = 0; wr < it.rg; ++wr) {
                 const int u0 = (it.t0 + kR * wr) * f.d + it.r0 + lc;
@@ -129,8 +145,16 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
                 }
                 if (o_lo >= o_hi) continue;
                 for (int s2 = 0; s2 < kR + f.len - 1; ++s2) {
-                    const int s = kR * wr + s2, k = s & 3;
-                    const int pos = t_elem_offset(it.cg, s, lc, it.box_rows);
+                    const int s = kR * wr + s2;
+                    const long long want = (long long)kTPadFront + (long long)(it.t0 + s) * f.d + it.r0 + lc;
+                    const bool in_series = want >= kTPadFront && want < kTPadFront + L;
+                    if ((s >> 2) < it.g_lo || (s >> 2) >= it.g_hi) {
+                        // a row the consumer skips: it must hold no sample
+                        REQUIRE(wide && !in_series, "a skipped row holds a sample");
+                        continue;
+                    }
+                    const int k = (s & 3) + (wide && lc >= kTWideCols ? 4 : 0);
+                    const int pos = wide ? t_wide_elem_offset(s, lc, it.box_rows, it.g_lo) : t_elem_offset(it.cg, s, lc, it.box_rows);
                     REQUIRE(pos >= 0 && pos < kTStageFloats, "read outside the stage");
                     if ((lc & 1) == 0) REQUIRE(pos % 2 == 0, "pair not 8-byte aligned");
                     // which sample the copy engine put there
@@ -139,9 +163,7 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
                     REQUIRE(rel >= 0 && j < it.box_rows, "read outside the box");
                     const long long y = ph[k].y + j;
                     const long long flat = y * run + ph[k].x + i + ph[k].j;
-                    const long long want = (long long)kTPadFront + (long long)(it.t0 + s) * f.d + it.r0 + lc;
                     REQUIRE(flat == want, "wrong sample: got flat %lld, want %lld", flat, want);
-                    const bool in_series = want >= kTPadFront && want < kTPadFront + L;
                     if (y < 0 || y >= ny) REQUIRE(!in_series, "zero fill where a sample is expected");
                 }
             }
@@ -151,9 +173,11 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
         for (int i = 0; i < plan.krec[fidx].nout; ++i)
             REQUIRE(cover[fidx][i] == 1, "kernel %d (len %d d %d p %d) output %d owned %d times", plan.krec[fidx].k,
                     plan.krec[fidx].len, plan.krec[fidx].d, plan.krec[fidx].p, i, (int)cover[fidx][i]);
-    std::printf("ok seed=%llu K=%d C=%d L=%d split=%d: %zu fast kernels, %zu generic, %zu S items, %zu T items\n",
+    size_t n_wide = 0;
+    for (const TItem& it : plan.titems) n_wide += it.wide != 0;
+    std::printf("ok seed=%llu K=%d C=%d L=%d split=%d: %zu fast kernels, %zu generic, %zu S items, %zu T items (%zu wide)\n",
                 (unsigned long long)seed, hp.K, hp.C, hp.L, plan.split, plan.krec.size(), plan.generic_list.size(),
-                plan.sitems.size(), plan.titems.size());
+                plan.sitems.size(), plan.titems.size(), n_wide);
     return 0;
 }
 
@@ -177,6 +201,7 @@ int main() {
     add(7, 166, 0); add(7, 166, 498); add(11, 99, 495); add(9, 7, 40); add(7, 64, 5); add(9, 65, 300); add(11, 100, 1);
     add(7, 1, 0); add(7, 1, 3); add(9, 63, 17); add(7, 127, 381); add(7, 128, 0); add(9, 124, 0); add(3, 5, 0); add(5, 70, 3);
     add(7, 129, 5); add(9, 77, 308); add(11, 91, 2);
+    add(7, 330, 990); add(7, 340, 1000); add(7, 512, 1536); add(11, 345, 1725);   // at most 16 rows of outputs: wide tiles
     rc |= check(0, hp.K, hp.C, hp.L, 64, &hp);
     return rc;
 }
