@@ -118,12 +118,25 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
             if (rest >= 2) { widths.push_back(2); rest -= 2; }
             if (rest >= 1) widths.push_back(1);
         };
-        // kernels whose outputs span at most 16 rows of A: wide tiles (8 column groups side by side,
-        // only the rows that hold samples), as long as two halves fit a stage
-        const int t_first = (int)tmin;
-        const TWindow win = t_window(t_first, kR + f.len - 1, f.d, hp.L);
-        const bool wide_ok = R16 == 1 && 2 * t_wide_half_floats(win.g_hi - win.g_lo) <= kTStageFloats;
+        // A single row group under 4-wide tiles would leave half of the warps idle: it can be cut into
+        // wide tiles instead (8 column groups side by side, only the rows that hold samples), as long
+        // as the two halves fit a stage.
+        auto wide_fits = [&](int r16) {
+            const TWindow win = t_window((int)(tmin + (int64_t)kR * r16), kR + f.len - 1, f.d, hp.L);
+            return C64 >= 5 && 2 * t_wide_half_floats(win.g_hi - win.g_lo) <= kTStageFloats;
+        };
+        std::vector<int> wide_widths(C64 / 8, 8);
+        {
+            int rest = C64 % 8;
+            if (rest >= 5) { wide_widths.push_back(8); rest = 0; }
+            if (rest >= 3) { wide_widths.push_back(4); rest = 0; }
+            if (rest >= 2) { wide_widths.push_back(2); rest -= 2; }
+            if (rest >= 1) wide_widths.push_back(1);
+        }
+        // candidates: main width 2, 4 or 1 over all row groups, or width 4 over an even number of row
+        // groups and wide tiles over the last one; the fewest block tiles win
         int best_cg = 2;
+        bool last_wide = false;
         int64_t best_tiles = INT64_MAX;
         for (int cg : {2, 4, 1}) {
             std::vector<int> widths;
@@ -132,56 +145,62 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
             for (int w : widths) tiles += (R16 + 8 / w - 1) / (8 / w);
             if (tiles < best_tiles) { best_tiles = tiles; best_cg = cg; }
         }
-        std::vector<int> widths;
-        if (wide_ok) {
-            widths.assign(C64 / 8, 8);
-            int rest = C64 % 8;
-            if (rest >= 5) { widths.push_back(8); rest = 0; }
-            if (rest >= 3) { widths.push_back(4); rest = rest > 4 ? rest - 4 : 0; }
-            if (rest >= 2) { widths.push_back(2); rest -= 2; }
-            if (rest >= 1) widths.push_back(1);
-        } else {
-            chunks_of(best_cg, widths);
+        if (R16 % 2 == 1 && wide_fits(R16 - 1)) {
+            std::vector<int> widths;
+            chunks_of(4, widths);
+            int64_t tiles = (int64_t)wide_widths.size();
+            for (int w : widths) tiles += (R16 - 1 + 8 / w - 1) / (8 / w);
+            if (tiles < best_tiles) { best_tiles = tiles; best_cg = 4; last_wide = true; }
         }
-        int c64 = 0;
-        for (int w : widths) {
-            const int rg_full = w == 8 ? 1 : 8 / w;
-            for (int r16 = 0; r16 < R16; r16 += rg_full) {
-                TItem it{};
-                it.rg = std::min(rg_full, R16 - r16);
-                it.wide = w == 8 ? 1 : 0;
-                it.cg = it.wide ? 4 : w;
-                it.t0 = (int32_t)(tmin + (int64_t)kR * r16); it.r0 = c64 * kWarpCols;
-                // a tile none of whose (row, column) pairs is an output of the kernel is left out
-                bool any_output = false;
-                for (int t = it.t0; t < it.t0 + kR * it.rg && !any_output; ++t) {
-                    const int64_t c_lo = std::max<int64_t>(it.r0, (int64_t)f.lo_u - (int64_t)t * f.d);
-                    const int64_t c_hi = std::min<int64_t>(std::min(it.r0 + kWarpCols * w, f.d), (int64_t)f.hi_u - (int64_t)t * f.d);
-                    any_output = c_lo < c_hi;
+        struct Band { int r16, nrg; std::vector<int> widths; };
+        std::vector<Band> bands;
+        std::vector<int> main_widths;
+        chunks_of(best_cg, main_widths);
+        const int main_rows = last_wide ? R16 - 1 : R16;
+        if (main_rows > 0) bands.push_back({0, main_rows, main_widths});
+        if (last_wide) bands.push_back({R16 - 1, 1, wide_widths});
+        for (const Band& band : bands) {
+            int c64 = 0;
+            for (int w : band.widths) {
+                const int rg_full = w == 8 ? 1 : 8 / w;
+                for (int r16 = band.r16; r16 < band.r16 + band.nrg; r16 += rg_full) {
+                    TItem it{};
+                    it.rg = std::min(rg_full, band.r16 + band.nrg - r16);
+                    it.wide = w == 8 ? 1 : 0;
+                    it.cg = it.wide ? 4 : w;
+                    it.t0 = (int32_t)(tmin + (int64_t)kR * r16); it.r0 = c64 * kWarpCols;
+                    // a tile none of whose (row, column) pairs is an output of the kernel is left out
+                    bool any_output = false;
+                    for (int t = it.t0; t < it.t0 + kR * it.rg && !any_output; ++t) {
+                        const int64_t c_lo = std::max<int64_t>(it.r0, (int64_t)f.lo_u - (int64_t)t * f.d);
+                        const int64_t c_hi = std::min<int64_t>(std::min(it.r0 + kWarpCols * w, f.d), (int64_t)f.hi_u - (int64_t)t * f.d);
+                        any_output = c_lo < c_hi;
+                    }
+                    if (!any_output) continue;
+                    it.d = f.d; it.len = f.len; it.m = f.m;
+                    const TWindow win = t_window(it.t0, kR + f.len - 1, f.d, hp.L);
+                    it.g_lo = it.wide ? win.g_lo : 0;
+                    it.g_hi = it.wide ? win.g_hi : t_box_rows(it.rg, f.len);
+                    it.box_rows = it.g_hi - it.g_lo;
+                    for (int q = 0; q < f.m; ++q) it.ch[q] = (uint8_t)f.ch[q];
+                    it.krec = ki;
+                    const auto key = std::make_tuple(f.d, t_box_cols(it.cg), it.box_rows);
+                    auto found = map_index.find(key);
+                    if (found == map_index.end()) {
+                        found = map_index.emplace(key, (int)out.tmaps.size()).first;
+                        out.tmaps.push_back({f.d, t_box_cols(it.cg), it.box_rows});
+                    }
+                    it.map = found->second;
+                    for (int ph = 0; ph < 4; ++ph) {
+                        const TPhase tp = t_phase(it.t0, it.r0, it.d, ph);
+                        it.x[ph] = tp.x; it.y[ph] = tp.y + it.g_lo; it.j[ph] = tp.j;
+                    }
+                    const double share = it.wide ? (double)it.box_rows / t_box_rows(1, f.len) : 1.0;
+                    out.tcost.push_back((double)f.m * (f.len * share + 2) + 8.0);
+                    out.titems.push_back(it);
                 }
-                if (!any_output) continue;
-                it.d = f.d; it.len = f.len; it.m = f.m;
-                it.g_lo = it.wide ? win.g_lo : 0;
-                it.g_hi = it.wide ? win.g_hi : t_box_rows(it.rg, f.len);
-                it.box_rows = it.g_hi - it.g_lo;
-                for (int q = 0; q < f.m; ++q) it.ch[q] = (uint8_t)f.ch[q];
-                it.krec = ki;
-                const auto key = std::make_tuple(f.d, t_box_cols(it.cg), it.box_rows);
-                auto found = map_index.find(key);
-                if (found == map_index.end()) {
-                    found = map_index.emplace(key, (int)out.tmaps.size()).first;
-                    out.tmaps.push_back({f.d, t_box_cols(it.cg), it.box_rows});
-                }
-                it.map = found->second;
-                for (int ph = 0; ph < 4; ++ph) {
-                    const TPhase tp = t_phase(it.t0, it.r0, it.d, ph);
-                    it.x[ph] = tp.x; it.y[ph] = tp.y + it.g_lo; it.j[ph] = tp.j;
-                }
-                const double share = it.wide ? (double)it.box_rows / t_box_rows(1, f.len) : 1.0;
-                out.tcost.push_back((double)f.m * (f.len * share + 2) + 8.0);
-                out.titems.push_back(it);
+                c64 += w;
             }
-            c64 += w;
         }
     }
     // every channel row of the zero-margined copy: front zeros, L samples, zeros for the run a box may
