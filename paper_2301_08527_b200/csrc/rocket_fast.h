@@ -91,6 +91,7 @@ ROCKET_CX int t_stage_floats(int rg, int cg, int len) { return 4 * t_phase_float
 ROCKET_CX int imax_cx(int a, int b) { return a > b ? a : b; }
 constexpr int kTStageFloats = imax_cx(imax_cx(t_stage_floats(8, 1, ROCKET_MAX_LENGTH), t_stage_floats(4, 2, ROCKET_MAX_LENGTH)),
                                       t_stage_floats(2, 4, ROCKET_MAX_LENGTH));
+constexpr int kTChunkTiles = 16;                                   // consecutive tiles a block draws at a time
 constexpr int kTWideCols = 256;                                    // columns of one half of a wide tile
 constexpr int kChunkExamples = 8;                                 // examples per pass through the fused kernels
 constexpr int kTPadFront = 128;                                    // zero floats before every channel row
@@ -119,7 +120,6 @@ struct PlanHost {
     std::vector<SBucket> sb;
     std::vector<SItem> sitems;
     std::vector<TItem> titems;            // kernel by kernel, in the order the blocks walk them
-    std::vector<double> tcost;            // relative cost of every T tile
     std::vector<TMapSpec> tmaps;          // tensor maps the T tiles refer to
     std::vector<int32_t> generic_list;    // kernels the fast path does not take
     int64_t pad_pitch = 0;                // floats per channel row of the zero-margined copy
@@ -131,14 +131,13 @@ struct PlanDevice {
     const SBucket* sb = nullptr;
     const SItem* sitems = nullptr;
     const TItem* titems = nullptr;
-    const int32_t* tranges = nullptr;     // [n_tblocks + 1]: block b walks T tiles [tranges[b], tranges[b+1]) of every example
     const int32_t* generic_list = nullptr;
-    unsigned* counters = nullptr;         // [0] S work counter
+    unsigned* counters = nullptr;         // [0] S work counter, [1] T work counter
     int* error_flag = nullptr;            // set when a bounded wait gave up
     const void* tmaps = nullptr;          // CUtensorMap[n_tmaps], 128 bytes each
     float* xpad = nullptr;                // zero-margined copy of the batch
     int64_t pad_pitch = 0;
-    int n_krec = 0, n_sitems = 0, n_titems = 0, n_generic = 0, n_tmaps = 0, n_tblocks = 0;
+    int n_krec = 0, n_sitems = 0, n_titems = 0, n_generic = 0, n_tmaps = 0;
 };
 
 // Builds the launch plan for the kernels in hp (host side, once per handle).

@@ -525,7 +525,7 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, int 
 // arrive on the stage's barrier, which releases them).
 struct TSlotItem {
     int32_t t0, r0, rg, cg, box_rows, rec_slot, wide, g_lo;
-    int32_t g_hi, pad_[3];
+    int32_t g_hi, n, stop, pad_;          // n: example of the tile; stop: no tile, the block is done
 };
 
 struct TShared {
@@ -616,21 +616,29 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    // every block walks the same slice of the tile list for every example in turn, so that all
-    // blocks read one example at a time (it stays in L2) and consecutive tiles share a kernel
-    const int i_beg = a.plan.tranges[blockIdx.x], i_end = a.plan.tranges[blockIdx.x + 1];
+    // Work is handed out in units of kTChunkTiles consecutive tiles of one example, example after
+    // example (all blocks read one example at a time, so it stays in L2; consecutive tiles mostly
+    // share a kernel).  The producer draws the units from a global counter and tells the consumers
+    // what to do through the ring, a stop item last.
+    const unsigned n_chunks = ((unsigned)a.plan.n_titems + kTChunkTiles - 1u) / kTChunkTiles;
+    const unsigned total_units = (unsigned)a.N * n_chunks;
     volatile int* abort_flag = &sh.abort;
 
     if (warp == kTConsumerWarps) {
         // ---- producer: one lane issues every copy of the block
-        if (lane == 0 && i_beg < i_end) {
+        if (lane == 0) {
             uint32_t st = 0, it = 0, nrec = 0;
             int cur_krec = -1;
             bool ok = true;
-            const int4* tp = reinterpret_cast<const int4*>(a.plan.titems + i_beg);
-            int4 w0 = __ldg(tp), w1 = __ldg(tp + 1), w2 = __ldg(tp + 2), w3 = __ldg(tp + 3), w4 = __ldg(tp + 4),
-                 w5 = __ldg(tp + 5), w6 = __ldg(tp + 6);
-            for (int n = 0; ok && n < a.N; ++n) {
+            unsigned u = atomicAdd(a.plan.counters + 1, 1u);
+            while (ok && u < total_units) {
+                const unsigned u_next = atomicAdd(a.plan.counters + 1, 1u);   // on its way while this unit is issued
+                const int n = (int)(u / n_chunks);
+                const int i_beg = (int)((u - (unsigned)n * n_chunks) * kTChunkTiles);
+                const int i_end = min(i_beg + (int)kTChunkTiles, a.plan.n_titems);
+                const int4* tp = reinterpret_cast<const int4*>(a.plan.titems + i_beg);
+                int4 w0 = __ldg(tp), w1 = __ldg(tp + 1), w2 = __ldg(tp + 2), w3 = __ldg(tp + 3), w4 = __ldg(tp + 4),
+                     w5 = __ldg(tp + 5), w6 = __ldg(tp + 6);
                 for (int i = i_beg; ok && i < i_end; ++i) {
                     if (*abort_flag) { ok = false; break; }
                     const int map = w0.x, t0 = w0.y, r0 = w0.z, rg = w0.w;
@@ -639,8 +647,7 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                     const int px[4] = {w4.x, w4.y, w4.z, w4.w}, py[4] = {w5.x, w5.y, w5.z, w5.w}, pj[4] = {w6.x, w6.y, w6.z, w6.w};
                     const int run = 4 * w1.x;
                     {   // the next tile's description is on its way while this one is issued
-                        int inext = i + 1;
-                        if (inext == i_end) inext = i_beg;
+                        const int inext = min(i + 1, i_end - 1);
                         tp = reinterpret_cast<const int4*>(a.plan.titems + inext);
                         w0 = __ldg(tp); w1 = __ldg(tp + 1); w2 = __ldg(tp + 2); w3 = __ldg(tp + 3); w4 = __ldg(tp + 4);
                         w5 = __ldg(tp + 5); w6 = __ldg(tp + 6);
@@ -664,7 +671,7 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                         if (q2 == 0) {
                             TSlotItem& si = sh.items[it % kTParamSlots];
                             si.t0 = t0; si.r0 = r0; si.rg = rg; si.cg = cg; si.box_rows = box_rows; si.rec_slot = (int)rslot;
-                            si.wide = wide; si.g_lo = g_lo; si.g_hi = g_hi;
+                            si.wide = wide; si.g_lo = g_lo; si.g_hi = g_hi; si.n = n; si.stop = 0;
                             if (new_rec) tx += (uint32_t)sizeof(KRec);
                         }
                         mbar_arrive_expect_tx(bar, tx);
@@ -686,6 +693,17 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                     }
                     ++it;
                 }
+                u = u_next;
+            }
+            if (ok) {   // the stop item takes a stage of its own (no copy)
+                const uint32_t slot = st % kTStages;
+                if (st >= (uint32_t)kTStages && !mbar_wait(empty0 + 8u * slot, ((st / kTStages) - 1u) & 1u)) {
+                    ok = false;
+                } else {
+                    sh.items[it % kTParamSlots].stop = 1;
+                    mbar_arrive(full0 + 8u * slot);
+                    ++st;
+                }
             }
             if (!ok) {
                 *abort_flag = 1;
@@ -702,8 +720,8 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
         // ---- consumers
         uint32_t st = 0, it = 0;
         bool ok = true;
-        for (int n = 0; ok && n < a.N; ++n) {
-            for (int i = i_beg; ok && i < i_end; ++i) {
+        for (;;) {
+            {
                 if (*abort_flag) { ok = false; break; }
                 const uint32_t slot = st % kTStages;
                 if (!mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) {
@@ -711,6 +729,8 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                     break;
                 }
                 const TSlotItem si = sh.items[it % kTParamSlots];
+                if (si.stop) break;
+                const int n = si.n;
                 const KRec* rec = recs + si.rec_slot;
                 const int t0 = si.t0, r0 = si.r0, rg = si.rg, cg = si.cg, box_rows = si.box_rows;
                 const int len = rec->len, d = rec->d, korig = rec->k;
@@ -939,52 +959,37 @@ __global__ void fast_bwd_finalize_kernel(const long long* __restrict__ accfix, c
 
 }  // namespace
 
+// Blocks of the T kernel: two per SM, never more than there are work units.
+static unsigned t_grid(int n_examples, int n_titems, int sms) {
+    const unsigned long long units = (unsigned long long)n_examples * ((n_titems + kTChunkTiles - 1) / kTChunkTiles);
+    return (unsigned)std::min<unsigned long long>(units, 2ull * (unsigned long long)sms);
+}
+
 cudaError_t upload_plan(FastState& fs) {
     const PlanHost& h = fs.host;
     PlanDevice& d = fs.dev;
     d = PlanDevice();
-    // the T tile list is cut into one slice of equal cost per block (two blocks per SM)
-    int dev = 0, sms = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
-    const int n_tblocks = h.titems.empty() ? 0 : (int)std::min<size_t>(h.titems.size(), (size_t)sms * 2);
-    std::vector<int32_t> tranges(n_tblocks + 1, 0);
-    if (n_tblocks > 0) {
-        double total_cost = 0.0;
-        for (double c : h.tcost) total_cost += c;
-        double run = 0.0;
-        int b = 1;
-        for (size_t i = 0; i < h.titems.size() && b < n_tblocks; ++i) {
-            run += h.tcost[i];
-            while (b < n_tblocks && run >= total_cost * b / n_tblocks) tranges[b++] = (int32_t)(i + 1);
-        }
-        for (; b <= n_tblocks; ++b) tranges[b] = (int32_t)h.titems.size();
-    }
     struct Part { const void* src; size_t bytes; size_t off; };
-    Part parts[8] = {
-        {tranges.data(), tranges.size() * 4, 0},
+    Part parts[7] = {
         {h.krec.data(), h.krec.size() * sizeof(KRec), 0},   {h.sb.data(), h.sb.size() * sizeof(SBucket), 0},
         {h.sitems.data(), h.sitems.size() * sizeof(SItem), 0}, {h.titems.data(), h.titems.size() * sizeof(TItem), 0},
         {h.generic_list.data(), h.generic_list.size() * 4, 0}, {nullptr, 256, 0}, {nullptr, 256, 0}};
     size_t total = 0;
     for (auto& pt : parts) { pt.off = total; total += align256(pt.bytes); }
-    e = cudaMalloc(&fs.plan_blob, std::max<size_t>(total, 256));
+    cudaError_t e = cudaMalloc(&fs.plan_blob, std::max<size_t>(total, 256));
     if (e != cudaSuccess) { fs.plan_blob = nullptr; return e; }
     char* base = static_cast<char*>(fs.plan_blob);
     e = cudaMemset(base, 0, std::max<size_t>(total, 256));
     for (auto& pt : parts)
         if (e == cudaSuccess && pt.src && pt.bytes) e = cudaMemcpy(base + pt.off, pt.src, pt.bytes, cudaMemcpyHostToDevice);
     if (e != cudaSuccess) { cudaFree(fs.plan_blob); fs.plan_blob = nullptr; return e; }
-    d.krec = reinterpret_cast<const KRec*>(base + parts[1].off);
-    d.sb = reinterpret_cast<const SBucket*>(base + parts[2].off);
-    d.sitems = reinterpret_cast<const SItem*>(base + parts[3].off);
-    d.titems = reinterpret_cast<const TItem*>(base + parts[4].off);
-    d.generic_list = reinterpret_cast<const int32_t*>(base + parts[5].off);
-    d.counters = reinterpret_cast<unsigned*>(base + parts[6].off);
-    d.error_flag = reinterpret_cast<int*>(base + parts[7].off);
-    d.tranges = reinterpret_cast<const int32_t*>(base + parts[0].off);
-    d.n_tblocks = n_tblocks;
+    d.krec = reinterpret_cast<const KRec*>(base + parts[0].off);
+    d.sb = reinterpret_cast<const SBucket*>(base + parts[1].off);
+    d.sitems = reinterpret_cast<const SItem*>(base + parts[2].off);
+    d.titems = reinterpret_cast<const TItem*>(base + parts[3].off);
+    d.generic_list = reinterpret_cast<const int32_t*>(base + parts[4].off);
+    d.counters = reinterpret_cast<unsigned*>(base + parts[5].off);
+    d.error_flag = reinterpret_cast<int*>(base + parts[6].off);
     d.n_krec = (int)h.krec.size(); d.n_sitems = (int)h.sitems.size(); d.n_titems = (int)h.titems.size();
     d.n_generic = (int)h.generic_list.size(); d.n_tmaps = (int)h.tmaps.size();
     d.pad_pitch = h.pad_pitch;
@@ -1120,8 +1125,9 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
         }
         if (fs.profile) cudaEventRecord(fs.evs[3 * c + 1], stream);
         if (pd.n_titems > 0) {
-            if (soft) fast_t_forward<1><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
-            else fast_t_forward<0><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
+            const unsigned grid = t_grid(nc, pd.n_titems, sms);
+            if (soft) fast_t_forward<1><<<grid, kTThreads, t_bytes, stream>>>(a);
+            else fast_t_forward<0><<<grid, kTThreads, t_bytes, stream>>>(a);
             count_launch();
         }
         if (fs.profile) {
@@ -1198,7 +1204,7 @@ cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t 
             count_launch();
         }
         if (pd.n_titems > 0) {
-            fast_t_forward<2><<<(unsigned)pd.n_tblocks, kTThreads, t_bytes, stream>>>(a);
+            fast_t_forward<2><<<t_grid(nc, pd.n_titems, sms), kTThreads, t_bytes, stream>>>(a);
             count_launch();
         }
     }

@@ -195,8 +195,6 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
                         const TPhase tp = t_phase(it.t0, it.r0, it.d, ph);
                         it.x[ph] = tp.x; it.y[ph] = tp.y + it.g_lo; it.j[ph] = tp.j;
                     }
-                    const double share = it.wide ? (double)it.box_rows / t_box_rows(1, f.len) : 1.0;
-                    out.tcost.push_back((double)f.m * (f.len * share + 2) + 8.0);
                     out.titems.push_back(it);
                 }
                 c64 += w;

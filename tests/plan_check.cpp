@@ -80,7 +80,6 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
 
     const int64_t pitch = plan.pad_pitch;
     REQUIRE(plan.titems.empty() || (pitch % 32 == 0 && pitch >= kTPadFront + L), "pad pitch");
-    REQUIRE(plan.tcost.size() == plan.titems.size(), "one cost per T tile");
     for (const TItem& it : plan.titems) {
         const KRec& f = plan.krec[it.krec];
         REQUIRE(it.map >= 0 && it.map < (int)plan.tmaps.size(), "T map index");
