@@ -91,7 +91,7 @@ ROCKET_CX int t_stage_floats(int rg, int cg, int len) { return 4 * t_phase_float
 ROCKET_CX int imax_cx(int a, int b) { return a > b ? a : b; }
 constexpr int kTStageFloats = imax_cx(imax_cx(t_stage_floats(8, 1, ROCKET_MAX_LENGTH), t_stage_floats(4, 2, ROCKET_MAX_LENGTH)),
                                       t_stage_floats(2, 4, ROCKET_MAX_LENGTH));
-constexpr int kTChunkTiles = 16;                                   // consecutive tiles a block draws at a time
+constexpr int kTChunkTiles = 4;                                    // consecutive tiles a block draws at a time
 constexpr int kTWideCols = 256;                                    // columns of one half of a wide tile
 constexpr int kChunkExamples = 8;                                 // examples per pass through the fused kernels
 constexpr int kTPadFront = 128;                                    // zero floats before every channel row
