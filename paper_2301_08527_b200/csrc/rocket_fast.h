@@ -93,7 +93,7 @@ constexpr int kTStageFloats = imax_cx(imax_cx(t_stage_floats(8, 1, ROCKET_MAX_LE
                                       t_stage_floats(2, 4, ROCKET_MAX_LENGTH));
 constexpr int kTChunkTiles = 4;                                    // consecutive tiles a block draws at a time
 constexpr int kTWideCols = 256;                                    // columns of one half of a wide tile
-constexpr int kChunkExamples = 8;                                 // examples per pass through the fused kernels
+constexpr int kChunkExamples = 12;                                // examples per pass through the fused kernels
 constexpr int kTPadFront = 128;                                    // zero floats before every channel row
 constexpr int kTXExtra = 256;                                      // floats a box may run past a 4d run
 
