@@ -35,7 +35,7 @@ LAMBDA, SHIFT = 10.0, 3.0
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the committed ncu capture
 # (profiles/); None until a capture of the current kernel exists.
-NCU_DRAM_BYTES_PER_LAUNCH = {"fast_s_forward": 38.3e6, "fast_t_forward": 827.5e6}   # per launch = one chunk of 8 examples
+NCU_DRAM_BYTES_PER_LAUNCH = {"fast_s_forward": None, "fast_t_forward": None}   # per launch = one chunk of 12 examples
 
 
 def fp32_peak_tflops(sm_count, sm_mhz):
@@ -184,7 +184,7 @@ def main():
     ap.add_argument("--skip-passes", action="store_true", help="skip the soft forward / backward timings")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="also time the throughput sweep (config 4) on rank 0")
-    ap.add_argument("--small", action="store_true", help="profiling case: N=8 examples (160 MB... of input)")
+    ap.add_argument("--small", action="store_true", help="profiling case: N=12 examples, one launch of either fused kernel")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -217,7 +217,7 @@ def main():
 
     w = dict(WORKLOAD)
     if args.small:
-        w["N"] = 8
+        w["N"] = 12
     props = torch.cuda.get_device_properties(local_rank)
     params = rk.RocketParams.generate(PARAM_SEED, w["K"], w["C"], w["L"])
     flops_ex, outputs_ex = params.work()
@@ -258,6 +258,9 @@ def main():
     clocks = sampler.stop() if sampler else None
     launches = rk.kernel_launch_count() - launches0
     launches_timed = launches * args.steps // (args.steps + args.warmup)
+    # one transform = init + per chunk of the batch (shifted copies, small-dilation kernel, large-dilation
+    # kernel) + finalise: the number of launches of either fused kernel per step follows from the count
+    chunk_launches = max(1, (launches // (args.steps + args.warmup) - 2) // 3)
     total_s = max_over(total_s)
     ms_per_step = 1e3 * total_s / args.steps
     value = whole_job_value(w["N"], args.steps, total_s, world)
@@ -293,8 +296,8 @@ def main():
     peak = fp32_peak_tflops(props.multi_processor_count, sm_max)
     roofline = {"bound": "alu", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(dom.split()[0]),
-                "launch_ms": dom_ms, "launches_per_step": (w["N"] + 7) // 8,
-                "traffic_note": "ncu, cold cache, one launch = one chunk of 8 examples (32 MB of input)",
+                "launch_ms": dom_ms, "launches_per_step": chunk_launches,
+                "traffic_note": "ncu, cold cache, one launch = one chunk of 12 examples (48 MB of input)",
                 "peak_source": "derived: %d SMs x 128 FP32 lanes x 2 flop x %.0f MHz (max SM clock from %s); "
                                "a packed-FMA microbenchmark reaches 74.0 TFLOP/s on this pool" % (
                                    props.multi_processor_count, sm_max,
