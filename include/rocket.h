@@ -160,6 +160,28 @@ int rocket_transform_soft_backward_host(rocket_params_t* p, const float* X_host,
                                         const int32_t* argmax_host, float* dW_host, float* db_host);
 
 /*
+ * The transform of raw 8-bit sensor intensities (Section 4.1: integer light intensities 0..255)
+ * under per-channel feature scaling (Section 4.3: every sensor channel is normalised on its own):
+ *     x[n][c][i] = ((float)X_u8[n][c][i] - mean[c]) * inv_std[c]      (two fp32 operations)
+ * followed by rocket_transform / rocket_transform_soft on x.  X_u8_dev is [N][C][L] bytes on the
+ * device; mean and inv_std are HOST arrays of C floats (statistics of the training set, not of the
+ * batch) and are read before the call returns; outputs, stream, ownership and errors as in the fp32
+ * forms, plus ROCKET_EINVAL for a NULL or NaN statistic.  When every kernel of the handle is served
+ * by the fused kernels (lengths 7/9/11, L % 4 == 0, C <= 20) and X_u8_dev is 4-byte aligned, the
+ * scaling happens while the kernels' staging copy of the batch is written and no fp32 copy of the
+ * batch exists; otherwise the call first writes a scaled fp32 copy into a buffer of the handle
+ * (grown with cudaMalloc on demand, ROCKET_ENOMEM if that fails) and takes the fp32 route.
+ * The host form copies the bytes to the device inside the call (a quarter of the fp32 form's traffic).
+ */
+int rocket_transform_u8(const rocket_params_t* p, const uint8_t* X_u8_dev, int N, int C, int L, const float* mean,
+                        const float* inv_std, float* feat_dev, void* cuda_stream);
+int rocket_transform_soft_u8(const rocket_params_t* p, const uint8_t* X_u8_dev, int N, int C, int L, const float* mean,
+                             const float* inv_std, float lambda, float shift, float* feat_dev, int32_t* argmax_dev,
+                             void* cuda_stream);
+int rocket_transform_u8_host(rocket_params_t* p, const uint8_t* X_u8_host, int N, int C, int L, const float* mean,
+                             const float* inv_std, float* feat_host);
+
+/*
  * Which kernels serve the handle: 0 = automatic (fast path where it applies), 1 = force the
  * generic kernels.  For tests and measurements; returns ROCKET_EINVAL for other values.
  */

@@ -92,6 +92,20 @@ def conv(p, X, n, k):
     return z
 
 
+def scale_u8(X_u8, mean, inv_std):
+    """Per-channel feature scaling of raw 8-bit intensities (Sections 4.1 and 4.3):
+    x[n, c, i] = (X_u8[n, c, i] - mean[c]) * inv_std[c], evaluated in float64 and rounded once to
+    the float32 input of the transform."""
+    v = np.asarray(X_u8)
+    if v.dtype != np.uint8 or v.ndim != 3:
+        raise ValueError("X_u8 must be a uint8 array [N, C, L]")
+    mean = np.asarray(mean, dtype=np.float64).reshape(1, -1, 1)
+    inv_std = np.asarray(inv_std, dtype=np.float64).reshape(1, -1, 1)
+    if mean.shape[1] != v.shape[1] or inv_std.shape[1] != v.shape[1]:
+        raise ValueError("one mean and one inv_std per channel")
+    return ((v.astype(np.float64) - mean) * inv_std).astype(np.float32)
+
+
 def forward_pairs(p, X, pair_n, pair_k, lam=1.0, shift=3.0, amb_eps=1e-5):
     """Pooled features for explicit (example, kernel) pairs.
 

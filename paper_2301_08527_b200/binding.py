@@ -48,6 +48,13 @@ SIGNATURES = {
                                                       ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_void_p,
                                                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                                       ctypes.c_void_p]),
+    "rocket_transform_u8": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "rocket_transform_soft_u8": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                                ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float,
+                                                ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "rocket_transform_u8_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                                ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "rocket_transform_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                                              ctypes.c_int, ctypes.c_void_p]),
     "rocket_transform_soft_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
@@ -239,6 +246,43 @@ def rocket_transform_soft(params, X, lam, shift=3.0, out=None, argmax_out=None, 
     return feat, arg
 
 
+def _stats(params, mean, inv_std):
+    m = np.ascontiguousarray(mean, dtype=np.float32)
+    s = np.ascontiguousarray(inv_std, dtype=np.float32)
+    if m.shape != (params.C,) or s.shape != (params.C,):
+        raise ValueError("mean and inv_std must hold one value per channel")
+    return m, s
+
+
+def rocket_transform_u8(params, X_u8, mean, inv_std, out=None):
+    """Hard PPV + max of raw 8-bit intensities scaled per channel: x = (v - mean[c]) * inv_std[c].
+    X_u8: CUDA uint8 [N, C, L]; mean, inv_std: host arrays of C floats."""
+    import torch
+    N, C, L = _check_x(params, X_u8)
+    m, s = _stats(params, mean, inv_std)
+    feat = out if out is not None else torch.empty((N, 2 * params.K), dtype=torch.float32, device=X_u8.device)
+    _check(load_library().rocket_transform_u8(params.handle, _dev_ptr(X_u8, torch.uint8, "X_u8"), N, C, L, _np_ptr(m),
+                                              _np_ptr(s), _dev_ptr(feat, torch.float32, "out"), _stream()),
+           "rocket_transform_u8")
+    return feat
+
+
+def rocket_transform_soft_u8(params, X_u8, mean, inv_std, lam, shift=3.0, out=None, argmax_out=None, want_argmax=True):
+    """softPPV + max of raw 8-bit intensities scaled per channel.  Returns (features, argmax or None)."""
+    import torch
+    N, C, L = _check_x(params, X_u8)
+    m, s = _stats(params, mean, inv_std)
+    feat = out if out is not None else torch.empty((N, 2 * params.K), dtype=torch.float32, device=X_u8.device)
+    arg = argmax_out
+    if arg is None and want_argmax:
+        arg = torch.empty((N, params.K), dtype=torch.int32, device=X_u8.device)
+    _check(load_library().rocket_transform_soft_u8(
+        params.handle, _dev_ptr(X_u8, torch.uint8, "X_u8"), N, C, L, _np_ptr(m), _np_ptr(s), ctypes.c_float(lam),
+        ctypes.c_float(shift), _dev_ptr(feat, torch.float32, "out"),
+        _dev_ptr(arg, torch.int32, "argmax_out") if arg is not None else None, _stream()), "rocket_transform_soft_u8")
+    return feat, arg
+
+
 def rocket_transform_soft_backward(params, X, lam, shift, dfeat, argmax, dW_out=None, db_out=None):
     """Gradients of sum(dfeat * soft features) for weights (ragged like the weights) and biases."""
     import torch
@@ -283,6 +327,17 @@ def rocket_transform_host(params, X_host, feat_host):
     _check(load_library().rocket_transform_host(params.handle, _host_ptr(X_host, torch.float32, "X_host"), N, C, L,
                                                 _host_ptr(feat_host, torch.float32, "feat_host")),
            "rocket_transform_host")
+    return feat_host
+
+
+def rocket_transform_u8_host(params, X_u8_host, mean, inv_std, feat_host):
+    """Host-buffer form of rocket_transform_u8 (the bytes travel to the device inside the call)."""
+    import torch
+    N, C, L = _check_x(params, X_u8_host)
+    m, s = _stats(params, mean, inv_std)
+    _check(load_library().rocket_transform_u8_host(params.handle, _host_ptr(X_u8_host, torch.uint8, "X_u8_host"), N, C, L,
+                                                   _np_ptr(m), _np_ptr(s), _host_ptr(feat_host, torch.float32, "feat_host")),
+           "rocket_transform_u8_host")
     return feat_host
 
 

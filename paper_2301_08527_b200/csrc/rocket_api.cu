@@ -248,6 +248,7 @@ void rocket_params_destroy(rocket_params_t* p) {
         if (p->dev_blob) cudaFree(p->dev_blob);
         if (p->fast) fast::release_fast_state(*p->fast);
         p->scratch.release();
+        p->u8_x.release(); p->u8_norm.release(); p->stage_u8.release();
         p->stage_x.release(); p->stage_feat.release(); p->stage_arg.release();
         p->stage_g.release(); p->stage_dw.release();
         if (p->host_stream) cudaStreamDestroy(p->host_stream);
@@ -356,6 +357,65 @@ int rocket_transform_soft(const rocket_params_t* p, const float* X_dev, int N, i
     return cuda_status(launch_generic_forward(p->dp, X_dev, N, true, lambda, shift, feat_dev, argmax_dev, stream));
 }
 
+// 8-bit input (Sections 4.1, 4.3): x = (v - mean[c]) * inv_std[c], then the transform of x.
+static int transform_u8(const rocket_params_t* p, const uint8_t* X_u8_dev, int N, int C, int L, const float* mean,
+                        const float* inv_std, bool soft, float lambda, float shift, float* feat_dev,
+                        int32_t* argmax_dev, void* cuda_stream) {
+    int st = check_call(p, X_u8_dev, N, C, L);
+    if (st != ROCKET_OK) return st;
+    if (!mean || !inv_std) return ROCKET_EINVAL;
+    for (int c = 0; c < C; ++c)
+        if (!(mean[c] == mean[c]) || !(inv_std[c] == inv_std[c])) return ROCKET_EINVAL;
+    if (soft && (!(lambda == lambda) || !(shift == shift))) return ROCKET_EINVAL;
+    if (N == 0) return ROCKET_OK;
+    if (!feat_dev) return ROCKET_EINVAL;
+    if ((st = ensure_device(p)) != ROCKET_OK) return st;
+    DeviceGuard g(p->device);
+    if (!g.ok) return ROCKET_ECUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const bool aligned = (reinterpret_cast<uintptr_t>(X_u8_dev) & 3u) == 0;
+    if (p->path == 0 && p->fast->host.enabled && p->fast->dev.n_generic == 0 && aligned && C <= fast::kNormMaxChannels) {
+        // every kernel is served by the fused kernels: the scaling happens while their staging copy is written
+        fast::NormArgs norm;
+        for (int c = 0; c < fast::kNormMaxChannels; ++c) {
+            norm.mean[c] = c < C ? mean[c] : 0.0f;
+            norm.inv_std[c] = c < C ? inv_std[c] : 0.0f;
+        }
+        return cuda_status(fast::launch_fast_forward(*p->fast, p->dp, nullptr, N, feat_dev, stream, soft, lambda, shift,
+                                                     argmax_dev, X_u8_dev, &norm));
+    }
+    // otherwise: a scaled fp32 copy of the batch in a buffer of the handle, then the fp32 route
+    const float* Xf = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(p->mu);
+        cudaError_t e = p->u8_x.reserve((size_t)N * C * L * sizeof(float));
+        if (e == cudaSuccess) e = p->u8_norm.reserve((size_t)2 * C * sizeof(float));
+        if (e != cudaSuccess) return cuda_status(e);
+        float* nb = static_cast<float*>(p->u8_norm.ptr);
+        // from pageable memory of the handle: the values are taken before the copy call returns
+        p->u8_norm_host.assign(mean, mean + C);
+        p->u8_norm_host.insert(p->u8_norm_host.end(), inv_std, inv_std + C);
+        e = cudaMemcpyAsync(nb, p->u8_norm_host.data(), (size_t)2 * C * sizeof(float), cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess)
+            e = launch_normalise_u8(X_u8_dev, (int64_t)N * C, L, C, nb, nb + C, static_cast<float*>(p->u8_x.ptr), stream);
+        if (e != cudaSuccess) return cuda_status(e);
+        Xf = static_cast<const float*>(p->u8_x.ptr);
+    }
+    return soft ? rocket_transform_soft(p, Xf, N, C, L, lambda, shift, feat_dev, argmax_dev, cuda_stream)
+                : rocket_transform(p, Xf, N, C, L, feat_dev, cuda_stream);
+}
+
+int rocket_transform_u8(const rocket_params_t* p, const uint8_t* X_u8_dev, int N, int C, int L, const float* mean,
+                        const float* inv_std, float* feat_dev, void* cuda_stream) {
+    return transform_u8(p, X_u8_dev, N, C, L, mean, inv_std, false, 0.0f, 0.0f, feat_dev, nullptr, cuda_stream);
+}
+
+int rocket_transform_soft_u8(const rocket_params_t* p, const uint8_t* X_u8_dev, int N, int C, int L, const float* mean,
+                             const float* inv_std, float lambda, float shift, float* feat_dev, int32_t* argmax_dev,
+                             void* cuda_stream) {
+    return transform_u8(p, X_u8_dev, N, C, L, mean, inv_std, true, lambda, shift, feat_dev, argmax_dev, cuda_stream);
+}
+
 int rocket_transform_soft_backward(const rocket_params_t* p, const float* X_dev, int N, int C, int L, float lambda,
                                    float shift, const float* dfeat_dev, const int32_t* argmax_dev, float* dW_dev,
                                    float* db_dev, void* cuda_stream) {
@@ -417,6 +477,29 @@ int rocket_transform_host(rocket_params_t* p, const float* X_host, int N, int C,
     ROCKET_TRY_CUDA(p->stage_feat.reserve(fb));
     ROCKET_TRY_CUDA(cudaMemcpyAsync(p->stage_x.ptr, X_host, xb, cudaMemcpyHostToDevice, s));
     st = rocket_transform(p, static_cast<const float*>(p->stage_x.ptr), N, C, L, static_cast<float*>(p->stage_feat.ptr), s);
+    if (st != ROCKET_OK) return st;
+    ROCKET_TRY_CUDA(cudaMemcpyAsync(feat_host, p->stage_feat.ptr, fb, cudaMemcpyDeviceToHost, s));
+    ROCKET_TRY_CUDA(cudaStreamSynchronize(s));
+    return ROCKET_OK;
+}
+
+int rocket_transform_u8_host(rocket_params_t* p, const uint8_t* X_u8_host, int N, int C, int L, const float* mean,
+                             const float* inv_std, float* feat_host) {
+    int st = check_call(p, X_u8_host, N, C, L);
+    if (st != ROCKET_OK) return st;
+    if (N == 0) return ROCKET_OK;
+    if (!feat_host) return ROCKET_EINVAL;
+    if ((st = ensure_device(p)) != ROCKET_OK) return st;
+    DeviceGuard g(p->device);
+    if (!g.ok) return ROCKET_ECUDA;
+    cudaStream_t s;
+    if ((st = host_stream_of(p, &s)) != ROCKET_OK) return st;
+    const size_t xb = (size_t)N * C * L, fb = (size_t)N * 2 * p->host.K * sizeof(float);
+    ROCKET_TRY_CUDA(p->stage_u8.reserve(xb));
+    ROCKET_TRY_CUDA(p->stage_feat.reserve(fb));
+    ROCKET_TRY_CUDA(cudaMemcpyAsync(p->stage_u8.ptr, X_u8_host, xb, cudaMemcpyHostToDevice, s));
+    st = rocket_transform_u8(p, static_cast<const uint8_t*>(p->stage_u8.ptr), N, C, L, mean, inv_std,
+                             static_cast<float*>(p->stage_feat.ptr), s);
     if (st != ROCKET_OK) return st;
     ROCKET_TRY_CUDA(cudaMemcpyAsync(feat_host, p->stage_feat.ptr, fb, cudaMemcpyDeviceToHost, s));
     ROCKET_TRY_CUDA(cudaStreamSynchronize(s));

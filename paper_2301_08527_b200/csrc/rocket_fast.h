@@ -63,6 +63,10 @@ static_assert(sizeof(KRec) == 128 + 4 * ROCKET_MAX_CHANNELS_PER_KERNEL * kPairRo
 static_assert(sizeof(KRec) % 16 == 0, "KRec must be copyable in 16-byte pieces");
 
 // ---- S regime --------------------------------------------------------------------------------
+// Per-channel feature scaling of 8-bit input (Section 4.3): x = (v - mean[c]) * inv_std[c].
+constexpr int kNormMaxChannels = 20;
+struct NormArgs { float mean[kNormMaxChannels], inv_std[kNormMaxChannels]; };
+
 constexpr int kSMaxChannels = 20;                                  // channels the S tile can stage
 constexpr int kSThreads = 512, kSWarps = kSThreads / 32;
 constexpr int kSPlaneFloats = kRowsMax * kWarpCols;                // one channel of an S tile
@@ -165,7 +169,7 @@ cudaError_t upload_plan(FastState& fs);
 // Frees everything upload_plan / ensure_pad_capacity allocated.
 void release_fast_state(FastState& fs);
 // Makes the padded copy hold N examples and (re-)encodes the tensor maps over it.
-cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L);
+cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L, bool without_maps = false);
 
 // Backward of the soft transform through the fast path (every kernel must be a fast-path kernel):
 // dW (ragged like the weights, n_weights floats) and db [K] are assigned.
@@ -175,9 +179,11 @@ cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t 
 
 // Forward through the fast path: init, pad copy, S kernel, T kernel, finalise.  soft = false:
 // PPV + max; soft = true: softPPV + max (+ argmax when argmax != nullptr).
+// With X_u8 (raw 8-bit intensities [N][C][L], 4-byte aligned) the samples are normalised per channel
+// with *norm while the zero-margined copies are written, and X is not read.
 cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const float* X, int N, float* feat,
                                 cudaStream_t stream, bool soft = false, float lambda = 0.0f, float shift = 0.0f,
-                                int32_t* argmax = nullptr);
+                                int32_t* argmax = nullptr, const uint8_t* X_u8 = nullptr, const NormArgs* norm = nullptr);
 
 }  // namespace fast
 }  // namespace rocket

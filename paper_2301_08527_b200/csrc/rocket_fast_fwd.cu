@@ -319,6 +319,7 @@ struct FwdArgs {
     const double* scale;     // [K] fixed-point scale of every kernel's sums
     long long n_weights;
     float lambda;
+    long long x_row_stride;  // floats between the channel rows of X (L, or the pitch of the zero-margined copy)
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -378,7 +379,7 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
         const SItem item = a.plan.sitems[g - (unsigned)n * n_items];
         const SBucket b = a.plan.sb[item.bucket];
         const int d = b.d;
-        const float* __restrict__ Xn = a.X + (size_t)n * a.C * a.L;
+        const float* __restrict__ Xn = a.X + (size_t)n * a.C * a.x_row_stride;
 
         // stage the tile: every channel, rows 0..rows-1 of every column, zero outside the series
         {
@@ -394,7 +395,7 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
 #pragma unroll 4
                 for (int c = 0; c < a.C; ++c) {
                     cp_async4_zfill(dst, src, ok);
-                    src += a.L;
+                    src += a.x_row_stride;
                     dst += kSPlaneFloats * 4;
                 }
             }
@@ -828,6 +829,30 @@ __global__ void fast_pad_copy_kernel(const float4* __restrict__ X, float* __rest
     }
 }
 
+// The same from raw 8-bit intensities (Section 4.1): every sample becomes (v - mean[c]) * inv_std[c]
+// (per-channel feature scaling, Section 4.3) on its way into the four copies.
+__global__ void fast_pad_copy_u8_kernel(const uchar4* __restrict__ X, float* __restrict__ xpad, int64_t rows, int L4,
+                                        int C, int64_t pitch, int front, int64_t copy_floats, NormArgs norm) {
+    const int64_t total = rows * L4;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t rho = e / L4;
+        const int i = (int)(e - rho * L4);
+        const int c = (int)(rho % C);
+        const uchar4 u = __ldg(X + e);
+        const float mu = norm.mean[c], is = norm.inv_std[c];
+        float4 v;
+        v.x = ((float)u.x - mu) * is; v.y = ((float)u.y - mu) * is;
+        v.z = ((float)u.z - mu) * is; v.w = ((float)u.w - mu) * is;
+        float* dst = xpad + rho * pitch + front + 4 * (int64_t)i;
+        *reinterpret_cast<float4*>(dst) = v;
+#pragma unroll
+        for (int j = 1; j < 4; ++j) {
+            float* dj = dst + j * copy_floats - j;
+            dj[0] = v.x; dj[1] = v.y; dj[2] = v.z; dj[3] = v.w;
+        }
+    }
+}
+
 __global__ void fast_init_kernel(int* __restrict__ feat_i, int64_t pairs, unsigned* counters) {
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e == 0) { counters[0] = 0u; counters[1] = 0u; }
@@ -1013,10 +1038,10 @@ void release_fast_state(FastState& fs) {
     fs.pad_examples = 0;
 }
 
-cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L) {
-    if (fs.host.tmaps.empty() || N <= fs.pad_examples) return cudaSuccess;
-    EncodeTiledFn encode = encode_tiled_fn();
-    if (!encode) return cudaErrorNotSupported;
+cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L, bool without_maps) {
+    if ((fs.host.tmaps.empty() && !without_maps) || N <= fs.pad_examples) return cudaSuccess;
+    EncodeTiledFn encode = fs.host.tmaps.empty() ? nullptr : encode_tiled_fn();
+    if (!encode && !fs.host.tmaps.empty()) return cudaErrorNotSupported;
     const int64_t pitch = fs.host.pad_pitch, rows = (int64_t)N * C;
     const int64_t copy_floats = (rows + 1) * pitch;   // pitch is a multiple of 32 floats
     const size_t bytes = (size_t)copy_floats * 4 * 4;
@@ -1042,12 +1067,14 @@ cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L) {
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
     static_assert(sizeof(CUtensorMap) == 128, "tensor maps are addressed in 128-byte steps");
-    if (!fs.maps_blob) {
-        e = cudaMalloc(&fs.maps_blob, n_maps * sizeof(CUtensorMap));
-        if (e != cudaSuccess) { fs.maps_blob = nullptr; return e; }
+    if (n_maps > 0) {
+        if (!fs.maps_blob) {
+            e = cudaMalloc(&fs.maps_blob, n_maps * sizeof(CUtensorMap));
+            if (e != cudaSuccess) { fs.maps_blob = nullptr; return e; }
+        }
+        e = cudaMemcpy(fs.maps_blob, maps.data(), n_maps * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) return e;
     }
-    e = cudaMemcpy(fs.maps_blob, maps.data(), n_maps * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
-    if (e != cudaSuccess) return e;
     fs.pad_examples = N;
     fs.copy_floats = copy_floats;
     fs.dev.tmaps = fs.maps_blob;
@@ -1056,7 +1083,8 @@ cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L) {
 }
 
 cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const float* X, int N, float* feat,
-                                cudaStream_t stream, bool soft, float lambda, float shift, int32_t* argmax) {
+                                cudaStream_t stream, bool soft, float lambda, float shift, int32_t* argmax,
+                                const uint8_t* X_u8, const NormArgs* norm) {
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -1066,8 +1094,8 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
     if (e != cudaSuccess) return e;
     const size_t s_bytes = s_smem_bytes(dp.C), t_bytes = t_smem_bytes();
     const PlanDevice& pd = fs.dev;
-    if (pd.n_titems > 0) {
-        e = ensure_pad_capacity(fs, std::min(N, kChunkExamples), dp.C, dp.L);
+    if (pd.n_titems > 0 || X_u8) {
+        e = ensure_pad_capacity(fs, std::min(N, kChunkExamples), dp.C, dp.L, X_u8 != nullptr);
         if (e != cudaSuccess) return e;
     }
     const int64_t pairs = (int64_t)N * dp.K;
@@ -1102,7 +1130,13 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
     }
     for (int c = 0; c < n_chunks; ++c) {
         const int n0 = c * kChunkExamples, nc = std::min(kChunkExamples, N - n0);
-        a.X = X + (size_t)n0 * dp.C * dp.L;
+        if (X_u8) {   // the kernels read the normalised samples from the unshifted zero-margined copy
+            a.X = fs.xpad + kTPadFront;
+            a.x_row_stride = fs.host.pad_pitch;
+        } else {
+            a.X = X + (size_t)n0 * dp.C * dp.L;
+            a.x_row_stride = dp.L;
+        }
         a.feat_i = feat_i + (size_t)n0 * 2 * dp.K;
         a.ws = ws ? ws + (size_t)n0 * 2 * dp.K : nullptr;
         a.N = nc;
@@ -1110,7 +1144,12 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
             e = cudaMemsetAsync(pd.counters, 0, 8, stream);
             if (e != cudaSuccess) return e;
         }
-        if (pd.n_titems > 0) {
+        if (X_u8) {
+            fast_pad_copy_u8_kernel<<<sms * 8, 256, 0, stream>>>(
+                reinterpret_cast<const uchar4*>(X_u8 + (size_t)n0 * dp.C * dp.L), fs.xpad, (int64_t)nc * dp.C, dp.L / 4, dp.C,
+                fs.host.pad_pitch, kTPadFront, fs.copy_floats, *norm);
+            count_launch();
+        } else if (pd.n_titems > 0) {
             fast_pad_copy_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(a.X), fs.xpad, (int64_t)nc * dp.C,
                                                               dp.L / 4, fs.host.pad_pitch, kTPadFront, fs.copy_floats);
             count_launch();
@@ -1184,6 +1223,7 @@ cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t 
     a.c1 = lambda * 1.4426950408889634f; a.c0 = -shift * 1.4426950408889634f;
     a.C = dp.C; a.L = dp.L; a.K = dp.K;
     a.accfix = accfix; a.scale = scale; a.n_weights = n_weights; a.lambda = lambda;
+    a.x_row_stride = dp.L;
     for (int n0 = 0; n0 < N; n0 += kChunkExamples) {
         const int nc = std::min(kChunkExamples, N - n0);
         a.X = X + (size_t)n0 * dp.C * dp.L;

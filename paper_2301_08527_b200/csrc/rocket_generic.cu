@@ -1,6 +1,7 @@
 // Generic kernels: one thread block per (example, kernel), inputs read straight from global
 // memory with a range test per tap.  They accept every kernel the handle accepts (any length
 // up to 11, any L, no alignment demands) and serve what the fast path does not cover.
+#include <algorithm>
 #include <cfloat>
 #include <climits>
 
@@ -185,7 +186,27 @@ reduce_examples_kernel(const float* __restrict__ scratch, int N, int64_t n_weigh
     else db[t - n_weights] = a;
 }
 
+// Per-channel feature scaling of raw 8-bit intensities (Sections 4.1 and 4.3).
+__global__ void __launch_bounds__(kThreads)
+normalise_u8_kernel(const uint8_t* __restrict__ X, int64_t total, int L, int C, const float* __restrict__ mean,
+                    const float* __restrict__ inv_std, float* __restrict__ out) {
+    for (int64_t e = (int64_t)blockIdx.x * kThreads + threadIdx.x; e < total; e += (int64_t)gridDim.x * kThreads) {
+        const int c = (int)((e / L) % C);
+        out[e] = ((float)X[e] - mean[c]) * inv_std[c];
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_normalise_u8(const uint8_t* X, int64_t rows, int L, int C, const float* mean, const float* inv_std,
+                                float* out, cudaStream_t stream) {
+    const int64_t total = rows * L;
+    if (total == 0) return cudaSuccess;
+    const unsigned grid = (unsigned)std::min<int64_t>((total + kThreads - 1) / kThreads, 148 * 16);
+    normalise_u8_kernel<<<grid, kThreads, 0, stream>>>(X, total, L, C, mean, inv_std, out);
+    count_launch();
+    return cudaGetLastError();
+}
 
 cudaError_t launch_generic_forward(const DeviceParams& dp, const float* X, int N, bool soft, float lambda,
                                    float shift, float* feat, int32_t* argmax, cudaStream_t stream,

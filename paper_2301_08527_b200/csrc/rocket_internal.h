@@ -49,6 +49,9 @@ cudaError_t launch_generic_forward(const DeviceParams& dp, const float* X, int N
                                    const int32_t* klist = nullptr, int nk = 0);
 // Backward: per-example partial gradients into scratch[N][nW + K], then a fixed-order sum over n.
 size_t generic_backward_scratch_floats(int N, int64_t n_weights, int K);
+// x[i] = (v[i] - mean[c]) * inv_std[c] for [rows][L] 8-bit samples, c = row % C (mean, inv_std on the device).
+cudaError_t launch_normalise_u8(const uint8_t* X, int64_t rows, int L, int C, const float* mean, const float* inv_std,
+                                float* out, cudaStream_t stream);
 cudaError_t launch_generic_backward(const DeviceParams& dp, int64_t n_weights, const float* X, int N,
                                     float lambda, float shift, const float* dfeat, const int32_t* argmax,
                                     float* scratch, float* dW, float* db, cudaStream_t stream);
@@ -81,7 +84,9 @@ struct rocket_params {
     mutable void* dev_blob = nullptr;  // one allocation holding every parameter array
     mutable rocket::DeviceParams dp{};
     mutable DeviceBuffer scratch; // backward partial sums
+    mutable DeviceBuffer u8_x, u8_norm;   // 8-bit input outside the fast path: normalised fp32 copy, mean / inv_std
+    mutable std::vector<float> u8_norm_host;
     rocket::fast::FastState* fast = nullptr;   // fast-path launch plan and its device-side state
-    DeviceBuffer stage_x, stage_feat, stage_arg, stage_g, stage_dw;  // host-call staging
+    DeviceBuffer stage_u8, stage_x, stage_feat, stage_arg, stage_g, stage_dw;  // host-call staging
     cudaStream_t host_stream = nullptr;
 };
