@@ -326,7 +326,27 @@ def main():
         s_bwd, _ = time_steps(lambda: rk.rocket_transform_soft_backward(params, Xt, LAMBDA, SHIFT, g, arg, dW, db),
                               psteps, 3)
         s_soft, s_bwd = max_over(s_soft) / psteps, max_over(s_bwd) / psteps
+        # the hard transform from raw 8-bit intensities (per-channel scaling fused into the staging copy):
+        # headline shape, device-resident bytes, and end to end from pinned host bytes
+        from rocket_inputs import channel_statistics, intensity_series_u8
+        X8_host = torch.from_numpy(intensity_series_u8(DATA_SEED + 1 + 1000 * rank, w["N"], w["C"], w["L"])).pin_memory()
+        mean8, istd8 = channel_statistics(X8_host.numpy()[:4])
+        X8 = X8_host.cuda()
+        s_u8, _ = time_steps(lambda: rk.rocket_transform_u8(params, X8, mean8, istd8, out=feat), psteps, 3)
+        s_u8 = max_over(s_u8) / psteps
+        for _ in range(2):
+            binding.rocket_transform_u8_host(params, X8_host, mean8, istd8, feat_host)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(psteps):
+            binding.rocket_transform_u8_host(params, X8_host, mean8, istd8, feat_host)
+        barrier()
+        s_u8_e2e = max_over(time.perf_counter() - t0) / psteps
+        del X8
         passes = {
+            "hard_u8": {"shape": "N=%d x C=%d x L=%d uint8, K=%d" % (w["N"], w["C"], w["L"], w["K"]),
+                        "examples_per_s": world * w["N"] / s_u8, "ms": 1e3 * s_u8,
+                        "e2e_examples_per_s": world * w["N"] / s_u8_e2e, "h2d_bytes_per_step": X8_host.numel()},
             "shape": "N=32 x C=20 x L=50000, K=10000 (config 3), lambda=%g, shift=%g" % (LAMBDA, SHIFT),
             "soft_forward": {"examples_per_s": world * t["N"] / s_soft, "ms": 1e3 * s_soft,
                              "conv_tflops": flops_ex * t["N"] / s_soft / 1e12},
