@@ -182,6 +182,30 @@ int rocket_transform_u8_host(rocket_params_t* p, const uint8_t* X_u8_host, int N
                              const float* inv_std, float* feat_host);
 
 /*
+ * The linear regressor on the pooled features (Section 3 step (3), Section 3.3: a ridge regressor on
+ * the 2K features of every example), fitted and applied on the device so that the features of the
+ * transform never leave it.
+ *
+ * rocket_ridge_fit: feat_dev [N][P] fp32 (row-major, P = 2K for the transform's output), y_dev [N]
+ * fp32 targets, alpha >= 0 the penalty on the weights.  The intercept is fitted and not penalised:
+ * with Fc, yc the column-centred features and targets, w minimises |Fc w - yc|^2 + alpha |w|^2 and
+ * b = mean(y) - mean(F) . w.  Solved in its dual form (an N x N system, N <= ROCKET_RIDGE_MAX_EXAMPLES)
+ * in double precision; w_dev [P] and b_dev [1] receive the result as fp32.  The call allocates its
+ * workspace ((P + N*N + N) doubles) with cudaMalloc, frees it, and returns after the work on
+ * cuda_stream has finished.  Errors: ROCKET_EINVAL for NULL pointers, N < 1, P < 1, a negative or
+ * non-finite alpha, or a system that is not positive definite (alpha = 0 with dependent rows);
+ * ROCKET_EUNSUPPORTED beyond the size limit; ROCKET_ENOMEM / ROCKET_ECUDA from the runtime.
+ *
+ * rocket_ridge_predict: yhat_dev[n] = b + sum_p feat_dev[n][p] w_dev[p] for n < N (products summed in
+ * double), enqueued on cuda_stream, no allocation.  All pointers are device pointers on the current device.
+ */
+#define ROCKET_RIDGE_MAX_EXAMPLES 4096
+int rocket_ridge_fit(const float* feat_dev, int N, int P, const float* y_dev, float alpha, float* w_dev, float* b_dev,
+                     void* cuda_stream);
+int rocket_ridge_predict(const float* feat_dev, int N, int P, const float* w_dev, const float* b_dev, float* yhat_dev,
+                         void* cuda_stream);
+
+/*
  * Which kernels serve the handle: 0 = automatic (fast path where it applies), 1 = force the
  * generic kernels.  For tests and measurements; returns ROCKET_EINVAL for other values.
  */

@@ -106,6 +106,27 @@ def scale_u8(X_u8, mean, inv_std):
     return ((v.astype(np.float64) - mean) * inv_std).astype(np.float32)
 
 
+def ridge_fit(F, y, alpha):
+    """Ridge regressor of Section 3.3 on features F [N, P] with targets y [N], float64 throughout:
+    the weights w minimise |Fc w - yc|^2 + alpha |w|^2 over the column-centred Fc, yc (the intercept
+    is not penalised), written out as the normal equations (Fc^T Fc + alpha I) w = Fc^T yc, and
+    b = mean(y) - mean(F) . w.  Returns (w [P], b)."""
+    F = np.asarray(F, dtype=np.float64)
+    y = np.asarray(y, dtype=np.float64)
+    if F.ndim != 2 or y.shape != (F.shape[0],):
+        raise ValueError("F must be [N, P] and y [N]")
+    mu, ybar = F.mean(axis=0), y.mean()
+    Fc, yc = F - mu, y - ybar
+    P = F.shape[1]
+    w = np.linalg.solve(Fc.T @ Fc + float(alpha) * np.eye(P), Fc.T @ yc)
+    return w, float(ybar - mu @ w)
+
+
+def ridge_predict(F, w, b):
+    """yhat = b + F w (Section 3 step (3)), float64."""
+    return np.asarray(F, dtype=np.float64) @ np.asarray(w, dtype=np.float64) + float(b)
+
+
 def forward_pairs(p, X, pair_n, pair_k, lam=1.0, shift=3.0, amb_eps=1e-5):
     """Pooled features for explicit (example, kernel) pairs.
 

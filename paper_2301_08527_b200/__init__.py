@@ -5,9 +5,11 @@ of librocket_b200.so.  There is no CPU fallback: importing works without a GPU (
 can be checked), but every compute call needs a CUDA device and the compiled library.
 """
 from .binding import (RocketError, RocketParams, kernel_launch_count, library_path, load_library,
+                      rocket_ridge_fit, rocket_ridge_predict,
                       rocket_transform, rocket_transform_soft, rocket_transform_soft_backward, rocket_transform_soft_u8,
                       rocket_transform_u8)
 
 __all__ = ["RocketError", "RocketParams", "kernel_launch_count", "library_path", "load_library",
+           "rocket_ridge_fit", "rocket_ridge_predict",
            "rocket_transform", "rocket_transform_soft", "rocket_transform_soft_backward", "rocket_transform_soft_u8",
            "rocket_transform_u8"]

@@ -55,6 +55,10 @@ SIGNATURES = {
                                                 ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "rocket_transform_u8_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                                                 ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "rocket_ridge_fit": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_float,
+                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "rocket_ridge_predict": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                            ctypes.c_void_p, ctypes.c_void_p]),
     "rocket_transform_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                                              ctypes.c_int, ctypes.c_void_p]),
     "rocket_transform_soft_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
@@ -309,6 +313,34 @@ def rocket_transform_soft_backward_noalloc(params, X, lam, shift, dfeat, argmax,
         _dev_ptr(dW_out, torch.float32, "dW_out"), _dev_ptr(db_out, torch.float32, "db_out"), _stream()),
         "rocket_transform_soft_backward_noalloc")
     return dW_out, db_out
+
+
+def rocket_ridge_fit(feat, y, alpha):
+    """Ridge regressor on pooled features (Section 3.3): feat CUDA fp32 [N, P], y CUDA fp32 [N].
+    Returns (w [P], b [1]) on the device; the intercept is fitted and not penalised."""
+    import torch
+    if feat.dim() != 2 or y.dim() != 1 or y.shape[0] != feat.shape[0]:
+        raise ValueError("feat must be [N, P] and y [N]")
+    N, Pn = int(feat.shape[0]), int(feat.shape[1])
+    w = torch.empty((Pn,), dtype=torch.float32, device=feat.device)
+    b = torch.empty((1,), dtype=torch.float32, device=feat.device)
+    _check(load_library().rocket_ridge_fit(_dev_ptr(feat, torch.float32, "feat"), N, Pn, _dev_ptr(y, torch.float32, "y"),
+                                           ctypes.c_float(alpha), _dev_ptr(w, torch.float32, "w"),
+                                           _dev_ptr(b, torch.float32, "b"), _stream()), "rocket_ridge_fit")
+    return w, b
+
+
+def rocket_ridge_predict(feat, w, b, out=None):
+    """yhat[n] = b + feat[n] . w on the device (current stream)."""
+    import torch
+    if feat.dim() != 2 or w.dim() != 1 or w.shape[0] != feat.shape[1]:
+        raise ValueError("feat must be [N, P] and w [P]")
+    N, Pn = int(feat.shape[0]), int(feat.shape[1])
+    yhat = out if out is not None else torch.empty((N,), dtype=torch.float32, device=feat.device)
+    _check(load_library().rocket_ridge_predict(_dev_ptr(feat, torch.float32, "feat"), N, Pn, _dev_ptr(w, torch.float32, "w"),
+                                               _dev_ptr(b, torch.float32, "b"), _dev_ptr(yhat, torch.float32, "out"),
+                                               _stream()), "rocket_ridge_predict")
+    return yhat
 
 
 def _host_ptr(t, dtype, name):
