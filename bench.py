@@ -343,7 +343,23 @@ def main():
         barrier()
         s_u8_e2e = max_over(time.perf_counter() - t0) / psteps
         del X8
+        # the regressor on the features (Section 3.3): fit at the size of the paper's training set, predict on
+        # the features of the timed batch
+        rngr = np.random.default_rng(GRAD_SEED)
+        Fr = torch.from_numpy(rngr.random((677, 2 * w["K"]), dtype=np.float32)).cuda()
+        yr = torch.from_numpy((0.6 + 1.2 * rngr.random(677)).astype(np.float32)).cuda()
+        rk.rocket_ridge_fit(Fr, yr, 1.0)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        wr, br = rk.rocket_ridge_fit(Fr, yr, 1.0)     # returns after its work has finished
+        s_fit = time.perf_counter() - t0
+        yhat = torch.empty((w["N"],), dtype=torch.float32, device="cuda")
+        s_pred, _ = time_steps(lambda: rk.rocket_ridge_predict(feat, wr, br, out=yhat), 5, 3)
+        s_pred /= 5
+        del Fr
         passes = {
+            "ridge": {"fit_ms": 1e3 * s_fit, "fit_shape": "677 examples x %d features, alpha=1" % (2 * w["K"]),
+                      "predict_ms": 1e3 * s_pred, "predict_shape": "%d examples x %d features" % (w["N"], 2 * w["K"])},
             "hard_u8": {"shape": "N=%d x C=%d x L=%d uint8, K=%d" % (w["N"], w["C"], w["L"], w["K"]),
                         "examples_per_s": world * w["N"] / s_u8, "ms": 1e3 * s_u8,
                         "e2e_examples_per_s": world * w["N"] / s_u8_e2e, "h2d_bytes_per_step": X8_host.numel()},
