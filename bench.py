@@ -35,7 +35,7 @@ LAMBDA, SHIFT = 10.0, 3.0
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the committed ncu capture
 # (profiles/); None until a capture of the current kernel exists.
-NCU_DRAM_BYTES_PER_LAUNCH = {"fast_s_forward": 56.4e6, "fast_t_forward": 313.4e6}   # per launch = one chunk of 12 examples
+NCU_DRAM_BYTES_PER_LAUNCH = {"fast_s_forward": 56.0e6, "fast_t_forward": 311.8e6}   # per launch = one chunk of 12 examples
 
 
 def fp32_peak_tflops(sm_count, sm_mhz):
