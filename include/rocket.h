@@ -206,6 +206,18 @@ int rocket_ridge_predict(const float* feat_dev, int N, int P, const float* w_dev
                          void* cuda_stream);
 
 /*
+ * Replaces the weights and biases of the handle's kernels (host arrays laid out as
+ * rocket_params_host_view returns them: n_weights ragged weights, K biases); lengths, dilations,
+ * paddings and channels stay.  This is the step that makes the kernels trainable (the paper's
+ * stated use of the soft PPV, Sections 1 and 6): rocket_transform_soft and
+ * rocket_transform_soft_backward give the loss gradient for the current values, the caller's
+ * optimiser produces new ones, this call installs them on the host and, if the handle is bound, on
+ * its device (it waits for the device first).  ROCKET_EINVAL for NULL or non-finite values (nothing
+ * is changed then).  Not to be called while another thread uses the handle.
+ */
+int rocket_params_set_weights(rocket_params_t* p, const float* weights, const float* bias);
+
+/*
  * Which kernels serve the handle: 0 = automatic (fast path where it applies), 1 = force the
  * generic kernels.  For tests and measurements; returns ROCKET_EINVAL for other values.
  */

@@ -30,6 +30,7 @@ SIGNATURES = {
                                           ctypes.POINTER(ctypes.c_double)]),
     "rocket_params_destroy": (None, [ctypes.c_void_p]),
     "rocket_params_set_path": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
+    "rocket_params_set_weights": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "rocket_params_bind_device": (ctypes.c_int, [ctypes.c_void_p]),
     "rocket_params_device_status": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int)]),
     "rocket_transform_soft_backward_noalloc": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
@@ -187,6 +188,14 @@ class RocketParams:
         _check(load_library().rocket_params_last_profile(self._h, *v), "rocket_params_last_profile")
         return {"ms_small_dilations": v[0].value, "ms_large_dilations": v[1].value,
                 "flops_small_dilations": v[2].value, "flops_large_dilations": v[3].value}
+
+    def set_weights(self, weights, bias):
+        """rocket_params_set_weights: install new weights (ragged, n_weights floats) and biases (K floats)."""
+        w = np.ascontiguousarray(weights, dtype=np.float32).reshape(-1)
+        b = np.ascontiguousarray(bias, dtype=np.float32).reshape(-1)
+        if w.shape[0] != self.n_weights or b.shape[0] != self.K:
+            raise ValueError("weights must hold n_weights values and bias K values")
+        _check(load_library().rocket_params_set_weights(self._h, _np_ptr(w), _np_ptr(b)), "rocket_params_set_weights")
 
     def set_path(self, path):
         _check(load_library().rocket_params_set_path(self._h, int(path)), "rocket_params_set_path")

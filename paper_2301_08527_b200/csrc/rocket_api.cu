@@ -272,6 +272,29 @@ int rocket_params_device_status(const rocket_params_t* p, int* wait_timeouts) {
     return cuda_status(cudaMemcpy(wait_timeouts, p->fast->dev.error_flag, sizeof(int), cudaMemcpyDeviceToHost));
 }
 
+int rocket_params_set_weights(rocket_params_t* p, const float* weights, const float* bias) {
+    if (!p || !weights || !bias) return ROCKET_EINVAL;
+    const size_t nw = p->host.weights.size(), nb = p->host.bias.size();
+    for (size_t i = 0; i < nw; ++i)
+        if (!(weights[i] - weights[i] == 0.0f)) return ROCKET_EINVAL;
+    for (size_t i = 0; i < nb; ++i)
+        if (!(bias[i] - bias[i] == 0.0f)) return ROCKET_EINVAL;
+    std::lock_guard<std::mutex> lk(p->mu);
+    p->host.weights.assign(weights, weights + nw);
+    p->host.bias.assign(bias, bias + nb);
+    if (p->fast)
+        for (fast::KRec& f : p->fast->host.krec) fast::fill_record_weights(p->host, f);
+    if (p->device < 0) return ROCKET_OK;
+    DeviceGuard g(p->device);
+    if (!g.ok) return ROCKET_ECUDA;
+    // work that still reads the old values finishes first
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess && nw) e = cudaMemcpy(const_cast<float*>(p->dp.weights), weights, nw * sizeof(float), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && nb) e = cudaMemcpy(const_cast<float*>(p->dp.bias), bias, nb * sizeof(float), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && p->fast) e = fast::upload_records(*p->fast);
+    return cuda_status(e);
+}
+
 int rocket_params_set_path(rocket_params_t* p, int path) {
     if (!p || path < 0 || path > 1) return ROCKET_EINVAL;
     p->path = path;

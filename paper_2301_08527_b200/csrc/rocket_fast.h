@@ -144,6 +144,11 @@ struct PlanDevice {
     int n_krec = 0, n_sitems = 0, n_titems = 0, n_generic = 0, n_tmaps = 0;
 };
 
+// Writes kernel f.k's bias and weights (negated, every weight twice) into its record.
+void fill_record_weights(const HostParams& hp, KRec& f);
+// Copies the records of the host plan to the device again (after their weights changed).
+cudaError_t upload_records(FastState& fs);
+
 // Builds the launch plan for the kernels in hp (host side, once per handle).
 void build_plan(const HostParams& hp, int split, PlanHost& out);
 

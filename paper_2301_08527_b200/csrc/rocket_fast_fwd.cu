@@ -1021,6 +1021,12 @@ cudaError_t upload_plan(FastState& fs) {
     return cudaSuccess;
 }
 
+cudaError_t upload_records(FastState& fs) {
+    if (!fs.plan_blob || fs.host.krec.empty()) return cudaSuccess;
+    return cudaMemcpy(const_cast<KRec*>(fs.dev.krec), fs.host.krec.data(), fs.host.krec.size() * sizeof(KRec),
+                      cudaMemcpyHostToDevice);
+}
+
 void release_fast_state(FastState& fs) {
     if (fs.plan_blob) cudaFree(fs.plan_blob);
     if (fs.maps_blob) cudaFree(fs.maps_blob);

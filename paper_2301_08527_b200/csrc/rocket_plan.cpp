@@ -15,6 +15,13 @@ inline int64_t floor_div(int64_t a, int64_t b) { return (a >= 0) ? a / b : -((-a
 
 }  // namespace
 
+void fill_record_weights(const HostParams& hp, KRec& f) {
+    const float* W = hp.weights.data() + hp.weight_offset[f.k];
+    f.negb = 0.0f - hp.bias[f.k];
+    for (int q = 0; q < f.m; ++q)
+        for (int j = 0; j < f.len; ++j) f.w2[q][2 * j] = f.w2[q][2 * j + 1] = 0.0f - W[q * f.len + j];
+}
+
 void build_plan(const HostParams& hp, int split, PlanHost& out) {
     out = PlanHost();
     out.flops_s = out.flops_t = 0.0;
@@ -40,16 +47,12 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         f.len = hp.length[k]; f.d = hp.dilation[k]; f.p = hp.padding[k]; f.m = hp.num_channels[k];
         f.nout = (int32_t)((int64_t)hp.L + 2 * (int64_t)f.p - (int64_t)(f.len - 1) * f.d);
         f.k = k; f.lo_u = -f.p; f.hi_u = f.nout - f.p;
-        f.negb = 0.0f - hp.bias[k];
         f.woff = hp.weight_offset[k];
         f.tl = (int32_t)floor_div(f.lo_u, f.d); f.rl = f.lo_u - f.tl * f.d;
         f.th = (int32_t)floor_div(f.hi_u, f.d); f.rh = f.hi_u - f.th * f.d;
         const int32_t* S = hp.channel_idx.data() + hp.channel_offset[k];
-        const float* W = hp.weights.data() + hp.weight_offset[k];
-        for (int q = 0; q < f.m; ++q) {
-            f.ch[q] = S[q];
-            for (int j = 0; j < f.len; ++j) f.w2[q][2 * j] = f.w2[q][2 * j + 1] = 0.0f - W[q * f.len + j];
-        }
+        for (int q = 0; q < f.m; ++q) f.ch[q] = S[q];
+        fill_record_weights(hp, f);
         out.krec.push_back(f);
     };
 

@@ -64,6 +64,24 @@ def _make(C, L, **kd):
     return rk.RocketParams.from_kernel_params(q)
 
 
+def test_set_weights_replaces_values_and_rejects_bad_input():
+    kp = generate_kernels(4, 50, 3, 200)
+    p = binding.RocketParams.from_kernel_params(kp)
+    w = (np.arange(p.n_weights, dtype=np.float32) * 0.01 - 1.0)
+    b = np.linspace(-0.5, 0.5, p.K).astype(np.float32)
+    p.set_weights(w, b)
+    arrs = p.host_arrays()
+    assert np.array_equal(arrs["weights"], w) and np.array_equal(arrs["bias"], b)
+    assert np.array_equal(arrs["dilation"], kp.dilation) and np.array_equal(arrs["channel_idx"], kp.channel_idx)
+    bad = w.copy(); bad[3] = np.inf
+    with pytest.raises(binding.RocketError):
+        p.set_weights(bad, b)
+    with pytest.raises(ValueError):
+        p.set_weights(w[:-1], b)
+    assert np.array_equal(p.host_arrays()["weights"], w)
+    p.close()
+
+
 def test_validation_rejects_bad_kernels():
     ok = dict(dilation=2, padding=0, channels=[0, 1], weights=np.ones((2, 7)), bias=0.0)
     _make(3, 100, **ok).close()
