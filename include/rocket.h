@@ -148,7 +148,8 @@ int rocket_transform_soft_backward(const rocket_params_t* p, const float* X_dev,
  * Host-buffer convenience forms of the three passes: inputs and outputs are HOST pointers
  * (pinned memory makes the copies asynchronous, pageable memory works too).  The call copies the inputs to
  * device buffers kept inside the handle (grown on demand, ROCKET_ENOMEM if that fails), runs
- * the pass, copies the results back and returns after they have arrived.  argmax_host may be
+ * the pass, copies the results back and returns after they have arrived (the forward forms upload
+ * the batch in chunks on a second stream of the handle and start on a chunk as soon as it is there).  argmax_host may be
  * NULL in the forward; it is required in the backward.  These calls mutate the handle's
  * staging buffers: one such call per handle at a time.
  */

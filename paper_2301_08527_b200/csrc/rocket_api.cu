@@ -1,6 +1,7 @@
 // C ABI of the ROCKET transform library: parameter handles, validation, dispatch.
 #include <algorithm>
 #include <cstring>
+#include <functional>
 #include <new>
 
 #include "rocket_fast.h"
@@ -252,6 +253,8 @@ void rocket_params_destroy(rocket_params_t* p) {
         p->stage_x.release(); p->stage_feat.release(); p->stage_arg.release();
         p->stage_g.release(); p->stage_dw.release();
         if (p->host_stream) cudaStreamDestroy(p->host_stream);
+        if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
+        for (cudaEvent_t ev : p->copy_events) cudaEventDestroy(ev);
         cudaGetLastError();
     }
     delete p->fast;
@@ -485,6 +488,49 @@ static int host_stream_of(rocket_params_t* p, cudaStream_t* s) {
         if (e__ != cudaSuccess) return cuda_status(e__);       \
     } while (0)
 
+// Host form of a forward transform, pipelined: the batch is uploaded on a second stream in chunks of
+// the size the fused kernels work through, and the transform of a chunk starts as soon as its bytes
+// have arrived, so all but the first upload hide behind the kernels.  run(n0, nc, stream) enqueues the
+// device transform of examples [n0, n0 + nc).
+static int host_pipeline(rocket_params_t* p, const void* X_host, size_t bytes_per_example, DeviceBuffer& stage, int N,
+                         float* feat_host, cudaStream_t s, const std::function<int(int, int, cudaStream_t)>& run) {
+    if (!p->copy_stream && cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking) != cudaSuccess) {
+        cudaGetLastError();
+        p->copy_stream = nullptr;
+        return ROCKET_ECUDA;
+    }
+    const int chunk = fast::kChunkExamples, n_chunks = (N + chunk - 1) / chunk;
+    while ((int)p->copy_events.size() < n_chunks) {
+        cudaEvent_t ev = nullptr;
+        ROCKET_TRY_CUDA(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+        p->copy_events.push_back(ev);
+    }
+    const size_t fb = (size_t)N * 2 * p->host.K * sizeof(float);
+    ROCKET_TRY_CUDA(stage.reserve((size_t)N * bytes_per_example));
+    ROCKET_TRY_CUDA(p->stage_feat.reserve(fb));
+    for (int c = 0; c < n_chunks; ++c) {
+        const int n0 = c * chunk, nc = std::min(chunk, N - n0);
+        const size_t off = (size_t)n0 * bytes_per_example;
+        ROCKET_TRY_CUDA(cudaMemcpyAsync(static_cast<char*>(stage.ptr) + off, static_cast<const char*>(X_host) + off,
+                                        (size_t)nc * bytes_per_example, cudaMemcpyHostToDevice, p->copy_stream));
+        ROCKET_TRY_CUDA(cudaEventRecord(p->copy_events[c], p->copy_stream));
+    }
+    int st = ROCKET_OK;
+    for (int c = 0; c < n_chunks && st == ROCKET_OK; ++c) {
+        const int n0 = c * chunk, nc = std::min(chunk, N - n0);
+        ROCKET_TRY_CUDA(cudaStreamWaitEvent(s, p->copy_events[c], 0));
+        st = run(n0, nc, s);
+    }
+    if (st != ROCKET_OK) {   // nothing of this call may still be in flight when it returns
+        cudaStreamSynchronize(p->copy_stream);
+        cudaStreamSynchronize(s);
+        return st;
+    }
+    ROCKET_TRY_CUDA(cudaMemcpyAsync(feat_host, p->stage_feat.ptr, fb, cudaMemcpyDeviceToHost, s));
+    ROCKET_TRY_CUDA(cudaStreamSynchronize(s));
+    return ROCKET_OK;
+}
+
 int rocket_transform_host(rocket_params_t* p, const float* X_host, int N, int C, int L, float* feat_host) {
     int st = check_call(p, X_host, N, C, L);
     if (st != ROCKET_OK) return st;
@@ -495,15 +541,12 @@ int rocket_transform_host(rocket_params_t* p, const float* X_host, int N, int C,
     if (!g.ok) return ROCKET_ECUDA;
     cudaStream_t s;
     if ((st = host_stream_of(p, &s)) != ROCKET_OK) return st;
-    const size_t xb = (size_t)N * C * L * sizeof(float), fb = (size_t)N * 2 * p->host.K * sizeof(float);
-    ROCKET_TRY_CUDA(p->stage_x.reserve(xb));
-    ROCKET_TRY_CUDA(p->stage_feat.reserve(fb));
-    ROCKET_TRY_CUDA(cudaMemcpyAsync(p->stage_x.ptr, X_host, xb, cudaMemcpyHostToDevice, s));
-    st = rocket_transform(p, static_cast<const float*>(p->stage_x.ptr), N, C, L, static_cast<float*>(p->stage_feat.ptr), s);
-    if (st != ROCKET_OK) return st;
-    ROCKET_TRY_CUDA(cudaMemcpyAsync(feat_host, p->stage_feat.ptr, fb, cudaMemcpyDeviceToHost, s));
-    ROCKET_TRY_CUDA(cudaStreamSynchronize(s));
-    return ROCKET_OK;
+    const size_t per_example = (size_t)C * L, K2 = (size_t)2 * p->host.K;
+    return host_pipeline(p, X_host, per_example * sizeof(float), p->stage_x, N, feat_host, s,
+                         [&](int n0, int nc, cudaStream_t stream) {
+                             return rocket_transform(p, static_cast<const float*>(p->stage_x.ptr) + n0 * per_example, nc, C, L,
+                                                     static_cast<float*>(p->stage_feat.ptr) + n0 * K2, stream);
+                         });
 }
 
 int rocket_transform_u8_host(rocket_params_t* p, const uint8_t* X_u8_host, int N, int C, int L, const float* mean,
@@ -517,16 +560,12 @@ int rocket_transform_u8_host(rocket_params_t* p, const uint8_t* X_u8_host, int N
     if (!g.ok) return ROCKET_ECUDA;
     cudaStream_t s;
     if ((st = host_stream_of(p, &s)) != ROCKET_OK) return st;
-    const size_t xb = (size_t)N * C * L, fb = (size_t)N * 2 * p->host.K * sizeof(float);
-    ROCKET_TRY_CUDA(p->stage_u8.reserve(xb));
-    ROCKET_TRY_CUDA(p->stage_feat.reserve(fb));
-    ROCKET_TRY_CUDA(cudaMemcpyAsync(p->stage_u8.ptr, X_u8_host, xb, cudaMemcpyHostToDevice, s));
-    st = rocket_transform_u8(p, static_cast<const uint8_t*>(p->stage_u8.ptr), N, C, L, mean, inv_std,
-                             static_cast<float*>(p->stage_feat.ptr), s);
-    if (st != ROCKET_OK) return st;
-    ROCKET_TRY_CUDA(cudaMemcpyAsync(feat_host, p->stage_feat.ptr, fb, cudaMemcpyDeviceToHost, s));
-    ROCKET_TRY_CUDA(cudaStreamSynchronize(s));
-    return ROCKET_OK;
+    const size_t per_example = (size_t)C * L, K2 = (size_t)2 * p->host.K;
+    return host_pipeline(p, X_u8_host, per_example, p->stage_u8, N, feat_host, s,
+                         [&](int n0, int nc, cudaStream_t stream) {
+                             return rocket_transform_u8(p, static_cast<const uint8_t*>(p->stage_u8.ptr) + n0 * per_example, nc, C,
+                                                        L, mean, inv_std, static_cast<float*>(p->stage_feat.ptr) + n0 * K2, stream);
+                         });
 }
 
 int rocket_transform_soft_host(rocket_params_t* p, const float* X_host, int N, int C, int L, float lambda,

@@ -89,4 +89,6 @@ struct rocket_params {
     rocket::fast::FastState* fast = nullptr;   // fast-path launch plan and its device-side state
     DeviceBuffer stage_u8, stage_x, stage_feat, stage_arg, stage_g, stage_dw;  // host-call staging
     cudaStream_t host_stream = nullptr;
+    cudaStream_t copy_stream = nullptr;        // host forms: uploads run ahead of the kernels on this stream
+    std::vector<cudaEvent_t> copy_events;      // one per chunk of a host-form call
 };
