@@ -188,6 +188,7 @@ int main() {
     rc |= check(12, 400, 7, 10000, 128);
     rc |= check(13, 300, 3, 1000, 64);
     rc |= check(14, 200, 2, 16, 64);
+    rc |= check(21, 300, 20, 200000, 64);
     // hand-made kernels: padding that is not a multiple of the dilation, extreme dilations, tiny outputs
     HostParams hp;
     hp.K = 0; hp.C = 2; hp.L = 1000;
