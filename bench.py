@@ -185,6 +185,8 @@ def main():
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="also time the throughput sweep (config 4) on rank 0")
     ap.add_argument("--small", action="store_true", help="profiling case: N=12 examples, one launch of either fused kernel")
+    ap.add_argument("--profile-pass", choices=["soft", "backward"], default=None,
+                    help="profiling case: run only that pass of config 3 on 12 examples, three times, and exit")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -228,6 +230,26 @@ def main():
     feat = torch.empty((w["N"], 2 * w["K"]), dtype=torch.float32, device="cuda")
     feat_host = torch.empty((w["N"], 2 * w["K"]), dtype=torch.float32).pin_memory()
     stream = torch.cuda.current_stream()
+
+    if args.profile_pass:
+        # one launch of either fused kernel per call: the case the ncu captures of the soft forward and
+        # of the backward use
+        Xs = X[:12].contiguous()
+        sfeat, arg = rk.rocket_transform_soft(params, Xs, LAMBDA, SHIFT)
+        g = torch.from_numpy(normal_array(GRAD_SEED, (12, 2 * w["K"]))).cuda()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for i in range(3):
+            if i == 2:
+                e0.record()
+            if args.profile_pass == "soft":
+                rk.rocket_transform_soft(params, Xs, LAMBDA, SHIFT, out=sfeat, argmax_out=arg)
+            else:
+                rk.rocket_transform_soft_backward(params, Xs, LAMBDA, SHIFT, g, arg)
+        e1.record()
+        torch.cuda.synchronize()
+        print(json.dumps({"pass": args.profile_pass, "shape": "N=12 x C=%d x L=%d, K=%d" % (w["C"], w["L"], w["K"]),
+                          "ms": e0.elapsed_time(e1)}))
+        return
 
     def time_steps(fn, steps, warmup, after_step=None):
         """CUDA-event time of `steps` calls on the launching stream, after `warmup` calls; seconds."""
