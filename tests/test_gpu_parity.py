@@ -236,6 +236,23 @@ def test_config4_sweep_points_hard_sampled(N, L, K):
     _check_sampled(kp, X, feat, pn, pk)
 
 
+def test_config4_largest_point_hard_sampled():
+    # the far corner of the sweep: 256 x 20 x 200,000 with 50,000 kernels (4 GB of input, built from eight
+    # generated examples repeated, one slot replaced by a fresh example)
+    N, L, K = 256, 200000, 50000
+    kp = generate_kernels(8527, K, 20, L)
+    X = np.concatenate([ar1_spike_series(2301, 8, 20, L)] * 32, axis=0)
+    X[200] = ar1_spike_series(99, 1, 20, L)[0]
+    feat = _run_hard(kp, X, 0)
+    _check_properties_hard(feat)
+    assert np.array_equal(feat[0], feat[8]) and np.array_equal(feat[3], feat[251])   # equal examples, equal rows
+    rng = np.random.default_rng(5)
+    ks = rng.choice(K, 150, replace=False)
+    pn = np.concatenate([np.full(150, 200), np.full(150, 255)]).astype(np.int32)
+    pk = np.concatenate([ks, ks]).astype(np.int32)
+    _check_sampled(kp, X, feat, pn, pk)
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_edge_cases(path):
     torch = _torch()
