@@ -76,7 +76,8 @@ int rocket_params_generate(uint64_t seed, int K, int C, int L, rocket_params_t**
  * Adopt caller-supplied kernels (the arrays are copied; the caller keeps ownership of its own).
  * Requirements, else ROCKET_EINVAL: 1 <= length[k] <= 11; dilation[k] >= 1; padding[k] >= 0;
  * L_out,k >= 1; 1 <= num_channels[k] <= min(C, 11); channel indices of one kernel distinct and
- * in [0, C).  Any such kernel is accepted; lengths 7, 9 and 11 take the fast path.
+ * in [0, C).  Any such kernel is accepted, up to L_out,k <= 2^30 (ROCKET_EUNSUPPORTED beyond);
+ * lengths 7, 9 and 11 take the fast path.
  */
 int rocket_params_from_arrays(int K, int C, int L, const int32_t* length, const int32_t* dilation,
                               const int32_t* padding, const int32_t* num_channels,
@@ -268,8 +269,12 @@ int64_t rocket_kernel_launch_count(void);
  *   - The handle must already be bound to its device (rocket_params_bind_device, or any
  *     earlier device call with it); binding allocates, so do it during set-up.  An unbound
  *     handle gives ROCKET_EINVAL.
- *   - The first call on each device looks up the array's device address (no allocation, but
- *     a runtime query); make that first call during set-up, before any stream capture.
+ *   - The first call on each device looks up the array's device address.  With the runtime's
+ *     lazy module loading that query, and the first launch of the kernels behind this call, may
+ *     load the library's device code onto the GPU, which allocates and synchronises inside the
+ *     driver.  So make one small call during set-up (N = 1 on any example will do: it runs the
+ *     look-up and both kernels), before any stream capture and before the phase that must not
+ *     allocate.
  *   - All calls on one device share the one array, and it keeps the previous call's contents.
  *     Nothing in it needs clearing: each call writes every element it later reads.  Two calls
  *     that overlap on the GPU (different streams, no event between them) race on it and give

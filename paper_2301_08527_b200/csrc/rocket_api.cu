@@ -28,7 +28,9 @@ int finish_host_params(HostParams& hp) {
         if (len < 1 || len > ROCKET_MAX_LENGTH || d < 1 || p < 0) return ROCKET_EINVAL;
         if (m < 1 || m > std::min<int64_t>(hp.C, ROCKET_MAX_CHANNELS_PER_KERNEL)) return ROCKET_EINVAL;
         const int64_t nout = (int64_t)hp.L + 2 * p - (len - 1) * d;
-        if (nout < 1 || nout > 0x7fffffffll || (len - 1) * d + 1 > 0x3fffffffll || p > 0x3fffffffll) return ROCKET_EINVAL;
+        if (nout < 1 || (len - 1) * d + 1 > 0x3fffffffll || p > 0x3fffffffll) return ROCKET_EINVAL;
+        // the kernels index outputs with 32-bit counters that step past the end by up to a block's width
+        if (nout > 0x40000000ll) return ROCKET_EUNSUPPORTED;
         co += m; wo += m * len;
         if (wo > 0x7fffffffll) return ROCKET_EUNSUPPORTED;
         hp.channel_offset[k + 1] = (int32_t)co;

@@ -68,24 +68,53 @@ constexpr int kNormMaxChannels = 20;
 struct NormArgs { float mean[kNormMaxChannels], inv_std[kNormMaxChannels]; };
 
 constexpr int kSMaxChannels = 20;                                  // channels the S tile can stage
-constexpr int kSThreads = 512, kSWarps = kSThreads / 32;
+#ifndef ROCKET_S_THREADS
+#define ROCKET_S_THREADS 512
+#endif
+constexpr int kSThreads = ROCKET_S_THREADS, kSWarps = kSThreads / 32;   // one block per SM
 constexpr int kSPlaneFloats = kRowsMax * kWarpCols;                // one channel of an S tile
 
 struct SBucket {
     int32_t d, tmin, nbands, raster_len;  // raster_len = nbands * d
     int32_t kbeg, kend, rows, pad_;       // kernels [kbeg, kend) of krec; rows = 16 + max len - 1
 };
-struct SItem { int32_t bucket, c0; };
+// One S tile: 64 raster positions from c0 of a bucket.  interior = 1 when every (row, column) of the
+// tile is an output of every kernel of the bucket (then the kernels need no range tests).
+struct SItem { int32_t bucket, c0, interior, pad_; };
 
 // ---- T regime --------------------------------------------------------------------------------
-constexpr int kTConsumerWarps = 8;
-constexpr int kTThreads = 32 * (kTConsumerWarps + 1);              // + one producer warp
-constexpr int kTStages = 2;
+// Consumer warps per block, blocks per SM and ring depth of the T kernel.  A block's consumer warps move
+// through a stage in step, so the number of independent blocks per SM decides how often the FMA pipes
+// find a warp that is ready.
+#ifndef ROCKET_T_WARPS
+#define ROCKET_T_WARPS 8
+#endif
+#ifndef ROCKET_T_BLOCKS
+#define ROCKET_T_BLOCKS 2
+#endif
+#ifndef ROCKET_T_STAGES
+#define ROCKET_T_STAGES 2
+#endif
+constexpr int kTConsumerWarps = ROCKET_T_WARPS;
+static_assert(kTConsumerWarps == 4 || kTConsumerWarps == 8, "tile shapes are laid out for 4 or 8 consumer warps");
+constexpr int kTBlocksPerSM = ROCKET_T_BLOCKS;
+constexpr int kTThreads = 32 * (kTConsumerWarps + 1);              // one group: consumer warps + one producer warp
+// Groups per block: every group is a producer with its consumers, its own ring and its own stream of tiles.
+// Two groups in one block instead of two blocks of one group leave more registers to every thread (the
+// register file is handed out per pair of warps, and a group has an odd number of warps).
+#ifndef ROCKET_T_GROUPS
+#define ROCKET_T_GROUPS 1
+#endif
+constexpr int kTGroups = ROCKET_T_GROUPS;
+constexpr int kTBlockThreads = kTGroups * kTThreads;
+constexpr int kTStages = ROCKET_T_STAGES;
 constexpr int kTParamSlots = kTStages + 2;
-// A T tile is rg row groups x cg column groups of warp tiles, rg * cg <= 8, cg in {1, 2, 4}.
+// A T tile is rg row groups x cg column groups of warp tiles, rg * cg <= the consumer warps, cg in {1, 2, 4}
+// (cg = 4 only with 8 consumer warps: a 16 x 256 tile would load 26 rows for 16 rows of outputs).
 // One box per phase brings all column groups (64 * cg floats wide).  The zero-margined copy is kept
 // four times, shifted by 0, 1, 2 and 3 floats, so that every row start is 16-byte aligned in one
 // of them: a box needs no alignment slack and every pair a consumer reads is 8-byte aligned.
+constexpr int kTMaxCg = kTConsumerWarps >= 8 ? 4 : 2;
 ROCKET_CX int t_box_cols(int cg) { return kWarpCols * cg; }
 // Box rows of one phase (rows s, s+4, ..), and the floats of one phase box (a multiple of 64
 // floats, so every box destination stays 128-byte aligned).
@@ -93,10 +122,12 @@ ROCKET_CX int t_box_rows(int rg, int len) { return (kR * rg + len - 1 + 3) / 4; 
 ROCKET_CX int t_phase_floats(int cg, int box_rows) { return box_rows * t_box_cols(cg); }
 ROCKET_CX int t_stage_floats(int rg, int cg, int len) { return 4 * t_phase_floats(cg, t_box_rows(rg, len)); }
 ROCKET_CX int imax_cx(int a, int b) { return a > b ? a : b; }
-constexpr int kTStageFloats = imax_cx(imax_cx(t_stage_floats(8, 1, ROCKET_MAX_LENGTH), t_stage_floats(4, 2, ROCKET_MAX_LENGTH)),
-                                      t_stage_floats(2, 4, ROCKET_MAX_LENGTH));
+constexpr int kTStageFloats =
+    imax_cx(imax_cx(t_stage_floats(kTConsumerWarps, 1, ROCKET_MAX_LENGTH), t_stage_floats(kTConsumerWarps / 2, 2, ROCKET_MAX_LENGTH)),
+            kTMaxCg >= 4 ? t_stage_floats(kTConsumerWarps / 4, 4, ROCKET_MAX_LENGTH) : 0);
 constexpr int kTChunkTiles = 4;                                    // consecutive tiles a block draws at a time
 constexpr int kTWideCols = 256;                                    // columns of one half of a wide tile
+constexpr int kTWideHalves = kTConsumerWarps / 4;                  // a wide tile is one row of all consumer warps' tiles
 constexpr int kChunkExamples = 12;                                // examples per pass through the fused kernels
 constexpr int kTPadFront = 128;                                    // zero floats before every channel row
 constexpr int kTXExtra = 256;                                      // floats a box may run past a 4d run
@@ -107,11 +138,13 @@ struct alignas(16) TItem {
     int32_t d, len, m, box_rows;
     uint8_t ch[12];
     int32_t krec;                         // index into the kernel records
-    int32_t cg, wide, g_lo, g_hi;         // wide tile: 1 x 8 warp tiles as two halves of 256 columns, of which only
+    int32_t cg, wide, g_lo, g_hi;         // wide tile: one row of warp tiles in halves of 256 columns, of which only
                                           // the groups of four rows [g_lo, g_hi) are loaded (box_rows = g_hi - g_lo)
     int32_t x[4], y[4];                   // tensor coordinates of the four phase boxes (first half; y of group g_lo)
     int32_t j[4];                         // which shifted copy each phase reads
-    int32_t pad1_[4];
+    // bit w: every output of consumer warp w's warp tile exists (no range tests needed) / at least one does
+    int32_t warp_interior, warp_active;
+    int32_t pad1_[2];
 };
 static_assert(sizeof(TItem) == 128, "TItem must be 32 words");
 // One tensor map: boxes of box_cols x box_rows floats over runs of 4 * d floats.

@@ -45,6 +45,11 @@ __device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
 __device__ __forceinline__ void fma2(u64& acc, u64 a, u64 b) {
     asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
 }
+__device__ __forceinline__ u64 fma2_to(u64 a, u64 b, u64 c) {
+    u64 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
 __device__ __forceinline__ float min3(float a, float b, float c) {
     float d;
     asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -62,10 +67,13 @@ __device__ __forceinline__ float key_float(int k) { return __int_as_float(k >= 0
 // streamed past them.  Row s of the tile sits at st[off[s & 3] + (s >> 2) * STEP]; w2 holds the
 // channel's negated weights, each twice.  With WIN, only the groups of four rows [gl, gh) are read
 // and multiplied (the others hold no sample and are not in shared memory); gl and gh are the same
-// for the whole warp.
-template <int ELL, int STEP, bool WIN>
+// for the whole warp.  With FIRST the accumulators come in undefined and every one of them starts as
+// init + w[0] * x (its first product), which is bit for bit what starting at init and adding gives.
+template <int ELL, int STEP, bool WIN, bool FIRST = false>
 __device__ __forceinline__ void conv_channel(const float* __restrict__ st, const int (&off)[4],
-                                             const float* __restrict__ w2, u64 (&acc)[kR], int gl = 0, int gh = 0) {
+                                             const float* __restrict__ w2, u64 (&acc)[kR], int gl = 0, int gh = 0,
+                                             u64 init = 0ull) {
+    static_assert(!(WIN && FIRST), "a windowed pass may skip an accumulator's first product");
     u64 wp[ELL + 1];
 #pragma unroll
     for (int j = 0; j < ELL; j += 2) {
@@ -83,14 +91,17 @@ __device__ __forceinline__ void conv_channel(const float* __restrict__ st, const
 #pragma unroll
                 for (int j = 0; j < ELL; ++j) {
                     const int o = s - j;
-                    if (o >= 0 && o < kR) fma2(acc[o], wp[j], x);
+                    if (o >= 0 && o < kR) {
+                        if (FIRST && j == 0) acc[o] = fma2_to(wp[0], x, init);
+                        else fma2(acc[o], wp[j], x);
+                    }
                 }
             }
         }
     }
 }
 
-// PPV count and min(-z) over the thread's 2 x 16 outputs.  Outputs outside the kernel's range
+// Adds the PPV count of the thread's 2 x 16 outputs to cnt and folds their min(-z) into mn.  Outputs outside the kernel's range
 // never need a test here: their accumulators start at +inf and stay there (sign bit clear,
 // neutral for the min).
 __device__ __forceinline__ void pool_hard(const u64 (&acc)[kR], int& cnt, float& mn) {
@@ -103,7 +114,7 @@ __device__ __forceinline__ void pool_hard(const u64 (&acc)[kR], int& cnt, float&
         signs = __funnelshift_l(__float_as_uint(b), signs, 1);
         mn = min3(mn, a, b);
     }
-    cnt = __popc(signs);
+    cnt += __popc(signs);
 }
 
 // Accumulators of a tile: 0 - bias where the output exists, +inf elsewhere.
@@ -350,11 +361,19 @@ __device__ __forceinline__ void s_grad_tile(const float* planes, const KRec* rec
     }
 }
 
+// The channels of one kernel on an S tile.  fold: the accumulators come in undefined and start at the
+// kernel's 0 - bias inside the first channel's pass (every output of the warp tile exists).
 template <int ELL>
-__device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* rec, int lane, u64 (&acc)[kR]) {
+__device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* rec, int lane, u64 (&acc)[kR], bool fold) {
     const int m = rec->m;
     const int off[4] = {2 * lane, kWarpCols + 2 * lane, 2 * kWarpCols + 2 * lane, 3 * kWarpCols + 2 * lane};
-    for (int q = 0; q < m; ++q)
+    int q = 0;
+    if (fold) {
+        const float nb = rec->negb;
+        conv_channel<ELL, 4 * kWarpCols, false, true>(planes + rec->ch[0] * kSPlaneFloats, off, rec->w2[0], acc, 0, 0, pack2(nb, nb));
+        q = 1;
+    }
+    for (; q < m; ++q)
         conv_channel<ELL, 4 * kWarpCols, false>(planes + rec->ch[q] * kSPlaneFloats, off, rec->w2[q], acc);
 }
 
@@ -379,6 +398,7 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
         const SItem item = a.plan.sitems[g - (unsigned)n * n_items];
         const SBucket b = a.plan.sb[item.bucket];
         const int d = b.d;
+        const bool tile_interior = item.interior != 0;
         const float* __restrict__ Xn = a.X + (size_t)n * a.C * a.x_row_stride;
 
         // stage the tile: every channel, rows 0..rows-1 of every column, zero outside the series
@@ -435,20 +455,25 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
             __syncwarp();
             const KRec* rec = myrec + cur;
             const int len = rec->len, korig = rec->k;
-            int lo0, hi0, lo1, hi1;
-            valid_rows_tc(trow0, c0, rec->tl, rec->rl, rec->th, rec->rh, kR, ok0, lo0, hi0);
-            valid_rows_tc(trow1, c1, rec->tl, rec->rl, rec->th, rec->rh, kR, ok1, lo1, hi1);
-            const bool interior = __all_sync(kFull, lo0 == 0 && lo1 == 0 && hi0 == kR && hi1 == kR);
+            // on an interior tile (the plan's flag) every output exists for every kernel of the bucket
+            int lo0 = 0, hi0 = kR, lo1 = 0, hi1 = kR;
+            bool interior = tile_interior;
+            if (!tile_interior) {
+                valid_rows_tc(trow0, c0, rec->tl, rec->rl, rec->th, rec->rh, kR, ok0, lo0, hi0);
+                valid_rows_tc(trow1, c1, rec->tl, rec->rl, rec->th, rec->rh, kR, ok1, lo1, hi1);
+                interior = __all_sync(kFull, lo0 == 0 && lo1 == 0 && hi0 == kR && hi1 == kR);
+            }
             u64 acc[kR];
-            init_acc(acc, rec->negb, interior, lo0, hi0, lo1, hi1);
-            if (len == 7) s_kernel_tile<7>(planes, rec, lane, acc);
-            else if (len == 9) s_kernel_tile<9>(planes, rec, lane, acc);
-            else s_kernel_tile<11>(planes, rec, lane, acc);
+            if (!interior) init_acc(acc, rec->negb, false, lo0, hi0, lo1, hi1);
+            if (len == 7) s_kernel_tile<7>(planes, rec, lane, acc, interior);
+            else if (len == 9) s_kernel_tile<9>(planes, rec, lane, acc, interior);
+            else s_kernel_tile<11>(planes, rec, lane, acc, interior);
             if (MODE == 2) {
                 const int64_t pair = (int64_t)n * a.K + korig;
                 const float gP = __ldg(a.dfeat + 2 * pair), gM = __ldg(a.dfeat + 2 * pair + 1);
                 const int uA = __ldg(a.argmax + pair) - rec->p;
-                const int tA = (uA + 8 * d) / d - 8, cA = uA - tA * d;   // uA >= -p > -8 d
+                int tA = uA / d, cA = uA - tA * d;                        // floor division: uA >= -p may be negative
+                if (cA < 0) { cA += d; --tA; }
                 const int oA0 = (ok0 && c0 == cA && tA >= trow0 && tA < trow0 + kR) ? tA - trow0 : -1;
                 const int oA1 = (ok1 && c1 == cA && tA >= trow1 && tA < trow1 + kR) ? tA - trow1 : -1;
                 float dbs = make_gz(acc, a.c1, a.c0, gP * a.lambda / (float)rec->nout, gM, interior, lo0, hi0, lo1, hi1, oA0, oA1);
@@ -526,8 +551,12 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, int 
 // arrive on the stage's barrier, which releases them).
 struct TSlotItem {
     int32_t t0, r0, rg, cg, box_rows, rec_slot, wide, g_lo;
-    int32_t g_hi, n, stop, pad_;          // n: example of the tile; stop: no tile, the block is done
+    int32_t g_hi, n, stop, flags;         // n: example of the tile; stop: no tile, the block is done;
+                                          // flags: the plan's warp_interior | warp_active << 8
 };
+
+// Dynamic shared memory of one group: the stages of its ring, then its kernel-record slots (a multiple of 128 bytes).
+constexpr size_t kTGroupSmemBytes = ((size_t)kTStages * kTStageFloats * 4 + (size_t)kTParamSlots * sizeof(KRec) + 127) / 128 * 128;
 
 struct TShared {
     unsigned long long full[kTStages];
@@ -541,12 +570,22 @@ struct TShared {
 template <int ELL, int STEP, bool WIN>
 __device__ __forceinline__ bool t_channels(const float* stages, const KRec* rec, const int (&off)[4], uint32_t full0,
                                            uint32_t empty0, uint32_t& st, int lane, bool active, u64 (&acc)[kR], int gl,
-                                           int gh) {
+                                           int gh, bool fold) {
     const int m = rec->m;
     for (int q = 0; q < m; ++q) {
         const uint32_t slot = st % kTStages;
         if (q > 0 && !mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) return false;
-        if (active) conv_channel<ELL, STEP, WIN>(stages + slot * kTStageFloats, off, rec->w2[q], acc, gl, gh);
+        if (active) {
+            bool done = false;
+            if constexpr (!WIN) {
+                if (fold && q == 0) {   // the accumulators start at 0 - bias inside the first channel's pass
+                    const float nb = rec->negb;
+                    conv_channel<ELL, STEP, false, true>(stages + slot * kTStageFloats, off, rec->w2[0], acc, 0, 0, pack2(nb, nb));
+                    done = true;
+                }
+            }
+            if (!done) conv_channel<ELL, STEP, WIN>(stages + slot * kTStageFloats, off, rec->w2[q], acc, gl, gh);
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * slot);
         ++st;
@@ -592,23 +631,26 @@ __device__ __forceinline__ bool t_grad_dispatch(int len, const float* stages, co
 template <int STEP, bool WIN>
 __device__ __forceinline__ bool t_dispatch(int len, const float* stages, const KRec* rec, const int (&off)[4],
                                            uint32_t full0, uint32_t empty0, uint32_t& st, int lane, bool active,
-                                           u64 (&acc)[kR], int gl, int gh) {
-    if (len == 7) return t_channels<7, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
-    if (len == 9) return t_channels<9, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
-    return t_channels<11, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
+                                           u64 (&acc)[kR], int gl, int gh, bool fold) {
+    if (len == 7) return t_channels<7, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh, fold);
+    if (len == 9) return t_channels<9, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh, fold);
+    return t_channels<11, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh, fold);
 }
 
 template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft
-__global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
-    __shared__ __align__(16) TShared sh;
-    // dynamic shared memory, aligned to 128 bytes by hand: stages, then kernel-record slots
+__global__ void __launch_bounds__(kTBlockThreads, kTBlocksPerSM) fast_t_forward(FwdArgs a) {
+    __shared__ __align__(16) TShared shs[kTGroups];
+    // the block's groups work independently of one another: each has its part of the shared memory
+    const int group = threadIdx.x / kTThreads, tid = threadIdx.x - group * kTThreads;
+    TShared& sh = shs[group];
+    // dynamic shared memory, aligned to 128 bytes by hand: per group its stages, then its kernel-record slots
     const uint32_t raw = smem_u32(smem_raw);
-    unsigned char* base = smem_raw + (((raw + 127u) & ~127u) - raw);
+    unsigned char* base = smem_raw + (((raw + 127u) & ~127u) - raw) + (size_t)group * kTGroupSmemBytes;
     float* stages = reinterpret_cast<float*>(base);
     KRec* recs = reinterpret_cast<KRec*>(base + (size_t)kTStages * kTStageFloats * 4);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = tid & 31, warp = tid >> 5;
     const uint32_t full0 = smem_u32(sh.full), empty0 = smem_u32(sh.empty);
-    if (threadIdx.x == 0) {
+    if (tid == 0) {
         for (int i = 0; i < kTStages; ++i) {
             mbar_init(full0 + 8u * i, 1);
             mbar_init(empty0 + 8u * i, kTConsumerWarps);
@@ -639,7 +681,7 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                 const int i_end = min(i_beg + (int)kTChunkTiles, a.plan.n_titems);
                 const int4* tp = reinterpret_cast<const int4*>(a.plan.titems + i_beg);
                 int4 w0 = __ldg(tp), w1 = __ldg(tp + 1), w2 = __ldg(tp + 2), w3 = __ldg(tp + 3), w4 = __ldg(tp + 4),
-                     w5 = __ldg(tp + 5), w6 = __ldg(tp + 6);
+                     w5 = __ldg(tp + 5), w6 = __ldg(tp + 6), w7 = __ldg(tp + 7);
                 for (int i = i_beg; ok && i < i_end; ++i) {
                     if (*abort_flag) { ok = false; break; }
                     const int map = w0.x, t0 = w0.y, r0 = w0.z, rg = w0.w;
@@ -647,11 +689,12 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                     const unsigned chw[3] = {(unsigned)w2.x, (unsigned)w2.y, (unsigned)w2.z};
                     const int px[4] = {w4.x, w4.y, w4.z, w4.w}, py[4] = {w5.x, w5.y, w5.z, w5.w}, pj[4] = {w6.x, w6.y, w6.z, w6.w};
                     const int run = 4 * w1.x;
+                    const int flags = (w7.x & 0xff) | ((w7.y & 0xff) << 8);
                     {   // the next tile's description is on its way while this one is issued
                         const int inext = min(i + 1, i_end - 1);
                         tp = reinterpret_cast<const int4*>(a.plan.titems + inext);
                         w0 = __ldg(tp); w1 = __ldg(tp + 1); w2 = __ldg(tp + 2); w3 = __ldg(tp + 3); w4 = __ldg(tp + 4);
-                        w5 = __ldg(tp + 5); w6 = __ldg(tp + 6);
+                        w5 = __ldg(tp + 5); w6 = __ldg(tp + 6); w7 = __ldg(tp + 7);
                     }
                     const uint32_t box_bytes = (uint32_t)box_rows * (uint32_t)t_box_cols(cg) * 4u;
                     const uint32_t phase_bytes = (uint32_t)t_phase_floats(cg, box_rows) * 4u;
@@ -668,11 +711,11 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                             break;
                         }
                         const uint32_t bar = full0 + 8u * slot;
-                        uint32_t tx = (wide ? 8u : 4u) * box_bytes;
+                        uint32_t tx = (wide ? 4u * (uint32_t)kTWideHalves : 4u) * box_bytes;
                         if (q2 == 0) {
                             TSlotItem& si = sh.items[it % kTParamSlots];
                             si.t0 = t0; si.r0 = r0; si.rg = rg; si.cg = cg; si.box_rows = box_rows; si.rec_slot = (int)rslot;
-                            si.wide = wide; si.g_lo = g_lo; si.g_hi = g_hi; si.n = n; si.stop = 0;
+                            si.wide = wide; si.g_lo = g_lo; si.g_hi = g_hi; si.n = n; si.stop = 0; si.flags = flags;
                             if (new_rec) tx += (uint32_t)sizeof(KRec);
                         }
                         mbar_arrive_expect_tx(bar, tx);
@@ -682,12 +725,14 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
                         const uint32_t dst0 = smem_u32(stages + slot * kTStageFloats);
 #pragma unroll
                         for (int k = 0; k < 4; ++k) tma_load_4d(dst0 + (uint32_t)k * phase_bytes, tmap, px[k], py[k], z, pj[k], bar);
-                        if (wide) {   // the second half: the boxes 256 columns further right
+                        if (wide) {   // the further halves: the boxes 256 columns further right each
+                            for (int h = 1; h < kTWideHalves; ++h) {
 #pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                int x2 = px[k] + kTWideCols, y2 = py[k];
-                                if (x2 >= run) { x2 -= run; ++y2; }
-                                tma_load_4d(dst0 + (uint32_t)(4 + k) * phase_bytes, tmap, x2, y2, z, pj[k], bar);
+                                for (int k = 0; k < 4; ++k) {
+                                    int x2 = px[k] + h * kTWideCols, y2 = py[k];
+                                    while (x2 >= run) { x2 -= run; ++y2; }
+                                    tma_load_4d(dst0 + (uint32_t)(4 * h + k) * phase_bytes, tmap, x2, y2, z, pj[k], bar);
+                                }
                             }
                         }
                         ++st;
@@ -721,84 +766,97 @@ __global__ void __launch_bounds__(kTThreads, 2) fast_t_forward(FwdArgs a) {
         // ---- consumers
         uint32_t st = 0, it = 0;
         bool ok = true;
+        // hard mode: the count and the min(-z) of the (example, kernel) pair the warp is working on travel from
+        // tile to tile (consecutive tiles mostly share a kernel) and are published when the pair changes
+        int64_t cur_pair = -1;
+        int cnt = 0;
+        float mn = __int_as_float(0x7f800000);
         for (;;) {
-            {
-                if (*abort_flag) { ok = false; break; }
-                const uint32_t slot = st % kTStages;
-                if (!mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) {
-                    ok = false;
-                    break;
-                }
-                const TSlotItem si = sh.items[it % kTParamSlots];
-                if (si.stop) break;
-                const int n = si.n;
-                const KRec* rec = recs + si.rec_slot;
-                const int t0 = si.t0, r0 = si.r0, rg = si.rg, cg = si.cg, box_rows = si.box_rows;
-                const int len = rec->len, d = rec->d, korig = rec->k;
-                const bool wide = si.wide != 0;
-                // warp tile (wr, wc) of the tile; a wide tile is one row of eight
-                const int wr = wide ? 0 : (cg == 1 ? warp : (cg == 2 ? warp >> 1 : warp >> 2));
-                const int wc = wide ? warp : (warp & (cg - 1));
-                const int lc = kWarpCols * wc + 2 * lane;
-                const bool in_tile = wr < rg;
-                const bool ok0 = in_tile && r0 + lc < d, ok1 = in_tile && r0 + lc + 1 < d;
-                int lo0, hi0, lo1, hi1;
+            if (*abort_flag) { ok = false; break; }
+            const uint32_t slot = st % kTStages;
+            if (!mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) {
+                ok = false;
+                break;
+            }
+            const TSlotItem si = sh.items[it % kTParamSlots];
+            if (si.stop) break;
+            const int n = si.n;
+            const KRec* rec = recs + si.rec_slot;
+            const int t0 = si.t0, r0 = si.r0, cg = si.cg, box_rows = si.box_rows;
+            const int len = rec->len, d = rec->d, korig = rec->k;
+            const bool wide = si.wide != 0;
+            // warp tile (wr, wc) of the tile; a wide tile is one row of all consumer warps' tiles
+            const int wr = wide ? 0 : (cg == 1 ? warp : (cg == 2 ? warp >> 1 : warp >> 2));
+            const int wc = wide ? warp : (warp & (cg - 1));
+            const int lc = kWarpCols * wc + 2 * lane;
+            // the plan says per warp whether every / any output of its warp tile exists
+            bool interior = ((si.flags >> warp) & 1) != 0;
+            const bool active = ((si.flags >> (8 + warp)) & 1) != 0;
+            const bool ok0 = active && r0 + lc < d, ok1 = active && r0 + lc + 1 < d;
+            int lo0 = 0, hi0 = kR, lo1 = 0, hi1 = kR;
+            if (active && !interior) {
                 valid_rows_tc(t0 + kR * wr, r0 + lc, rec->tl, rec->rl, rec->th, rec->rh, kR, ok0, lo0, hi0);
                 valid_rows_tc(t0 + kR * wr, r0 + lc + 1, rec->tl, rec->rl, rec->th, rec->rh, kR, ok1, lo1, hi1);
-                const bool interior = __all_sync(kFull, lo0 == 0 && lo1 == 0 && hi0 == kR && hi1 == kR);
-                const bool active = __any_sync(kFull, lo0 < hi0 || lo1 < hi1);
-                const int boxw = t_box_cols(cg);
-                int off[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    off[k] = wide ? t_wide_elem_offset(k, lc, box_rows, si.g_lo)
-                                  : t_box_offset(cg, k, box_rows) + 4 * wr * boxw + lc;
-                const int gl = si.g_lo, gh = si.g_hi;
-                u64 acc[kR];
-                init_acc(acc, rec->negb, interior, lo0, hi0, lo1, hi1);
-                if (wide) ok = t_dispatch<kTWideCols, true>(len, stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
-                else if (cg == 1) ok = t_dispatch<kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
-                else if (cg == 2) ok = t_dispatch<2 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
-                else ok = t_dispatch<4 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
-                if (!ok) break;
-                if (MODE == 2) {
-                    const int64_t pair = (int64_t)n * a.K + korig;
-                    double scale = 0.0;
-                    if (active) {
-                        const float gP = __ldg(a.dfeat + 2 * pair), gM = __ldg(a.dfeat + 2 * pair + 1);
-                        const int uA = __ldg(a.argmax + pair) - rec->p;
-                        const int tA = (uA + 8 * d) / d - 8, cA = uA - tA * d;   // uA >= -p > -8 d
-                        const int trow = t0 + kR * wr, c0 = r0 + lc;
-                        const bool rowhit = tA >= trow && tA < trow + kR;
-                        const int oA0 = (ok0 && rowhit && c0 == cA) ? tA - trow : -1;
-                        const int oA1 = (ok1 && rowhit && c0 + 1 == cA) ? tA - trow : -1;
-                        float dbs = make_gz(acc, a.c1, a.c0, gP * a.lambda / (float)rec->nout, gM, interior, lo0, hi0, lo1, hi1, oA0,
-                                            oA1);
-#pragma unroll
-                        for (int sh = 16; sh > 0; sh >>= 1) dbs += __shfl_xor_sync(kFull, dbs, sh);
-                        scale = __ldg(a.scale + korig);
-                        if (lane == 0) add_fixed(a.accfix + a.n_weights + korig, dbs, scale);
-                    }
-                    if (wide) ok = t_grad_dispatch<kTWideCols, true>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale, gl, gh);
-                    else if (cg == 1) ok = t_grad_dispatch<kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale, 0, 0);
-                    else if (cg == 2) ok = t_grad_dispatch<2 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale, 0, 0);
-                    else ok = t_grad_dispatch<4 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale, 0, 0);
-                    if (!ok) break;
-                } else if (active) {
-                    if (MODE == 1) {
-                        const int base = (t0 + kR * wr) * d + r0 + lc + rec->p;
-                        pool_publish_soft(a.ws, (int64_t)n * a.K + korig, acc, a.c1, a.c0, interior, lo0, hi0, lo1, hi1, base,
-                                          base + 1, d, lane);
-                    } else {
-                        int cnt = 0;
-                        float mn = __int_as_float(0x7f800000);
-                        pool_hard(acc, cnt, mn);
-                        publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
-                    }
-                }
-                ++it;
             }
+            const int boxw = t_box_cols(cg);
+            int off[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                off[k] = wide ? t_wide_elem_offset(k, lc, box_rows, si.g_lo)
+                              : t_box_offset(cg, k, box_rows) + 4 * wr * boxw + lc;
+            const int gl = si.g_lo, gh = si.g_hi;
+            u64 acc[kR];
+            // interior warp tiles of ordinary tiles start their accumulators inside the first channel's pass
+            const bool fold = interior && !wide;
+            if (active && !fold) init_acc(acc, rec->negb, interior, lo0, hi0, lo1, hi1);
+            if (wide) ok = t_dispatch<kTWideCols, true>(len, stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh, false);
+            else if (cg == 1) ok = t_dispatch<kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0, fold);
+            else if (cg == 2) ok = t_dispatch<2 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0, fold);
+            else ok = t_dispatch<4 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0, fold);
+            if (!ok) break;
+            const int64_t pair = (int64_t)n * a.K + korig;
+            if (MODE == 2) {
+                double scale = 0.0;
+                if (active) {
+                    const float gP = __ldg(a.dfeat + 2 * pair), gM = __ldg(a.dfeat + 2 * pair + 1);
+                    const int uA = __ldg(a.argmax + pair) - rec->p;
+                    int tA = uA / d, cA = uA - tA * d;                        // floor division: uA >= -p may be negative
+                    if (cA < 0) { cA += d; --tA; }
+                    const int trow = t0 + kR * wr, c0 = r0 + lc;
+                    const bool rowhit = tA >= trow && tA < trow + kR;
+                    const int oA0 = (ok0 && rowhit && c0 == cA) ? tA - trow : -1;
+                    const int oA1 = (ok1 && rowhit && c0 + 1 == cA) ? tA - trow : -1;
+                    float dbs = make_gz(acc, a.c1, a.c0, gP * a.lambda / (float)rec->nout, gM, interior, lo0, hi0, lo1, hi1, oA0,
+                                        oA1);
+#pragma unroll
+                    for (int sh = 16; sh > 0; sh >>= 1) dbs += __shfl_xor_sync(kFull, dbs, sh);
+                    scale = __ldg(a.scale + korig);
+                    if (lane == 0) add_fixed(a.accfix + a.n_weights + korig, dbs, scale);
+                }
+                if (wide) ok = t_grad_dispatch<kTWideCols, true>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale, gl, gh);
+                else if (cg == 1) ok = t_grad_dispatch<kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale, 0, 0);
+                else if (cg == 2) ok = t_grad_dispatch<2 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale, 0, 0);
+                else ok = t_grad_dispatch<4 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, a.accfix, scale, 0, 0);
+                if (!ok) break;
+            } else if (active) {
+                if (MODE == 1) {
+                    const int base = (t0 + kR * wr) * d + r0 + lc + rec->p;
+                    pool_publish_soft(a.ws, pair, acc, a.c1, a.c0, interior, lo0, hi0, lo1, hi1, base, base + 1, d, lane);
+                } else {
+                    if (pair != cur_pair) {
+                        if (cur_pair >= 0) publish(a.feat_i, cur_pair, cnt, mn, lane);
+                        cur_pair = pair;
+                        cnt = 0;
+                        mn = __int_as_float(0x7f800000);
+                    }
+                    pool_hard(acc, cnt, mn);
+                }
+            }
+            ++it;
         }
+        // what the warp still carries is published even when a wait gave up: counts and maxima are only
+        // ever combined with commutative atomics, and the error flag marks the result as incomplete
+        if (MODE == 0 && cur_pair >= 0) publish(a.feat_i, cur_pair, cnt, mn, lane);
         if (!ok) {
             *abort_flag = 1;
             if (lane == 0) atomicExch(a.plan.error_flag, 1);
@@ -894,7 +952,7 @@ __global__ void fast_finalize_soft_kernel(float* __restrict__ feat, int32_t* __r
 size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 size_t s_smem_bytes(int C) { return (size_t)C * kSPlaneFloats * 4 + (size_t)kSWarps * 2 * sizeof(KRec); }
-size_t t_smem_bytes() { return (size_t)kTStages * kTStageFloats * 4 + (size_t)kTParamSlots * sizeof(KRec) + 128; }
+size_t t_smem_bytes() { return (size_t)kTGroups * kTGroupSmemBytes + 128; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -984,10 +1042,10 @@ __global__ void fast_bwd_finalize_kernel(const long long* __restrict__ accfix, c
 
 }  // namespace
 
-// Blocks of the T kernel: two per SM, never more than there are work units.
+// Blocks of the T kernel: as many as are resident at a time, never more than there are work units.
 static unsigned t_grid(int n_examples, int n_titems, int sms) {
     const unsigned long long units = (unsigned long long)n_examples * ((n_titems + kTChunkTiles - 1) / kTChunkTiles);
-    return (unsigned)std::min<unsigned long long>(units, 2ull * (unsigned long long)sms);
+    return (unsigned)std::min<unsigned long long>((units + kTGroups - 1) / kTGroups, (unsigned long long)kTBlocksPerSM * (unsigned long long)sms);
 }
 
 cudaError_t upload_plan(FastState& fs) {
@@ -1171,8 +1229,8 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
         if (fs.profile) cudaEventRecord(fs.evs[3 * c + 1], stream);
         if (pd.n_titems > 0) {
             const unsigned grid = t_grid(nc, pd.n_titems, sms);
-            if (soft) fast_t_forward<1><<<grid, kTThreads, t_bytes, stream>>>(a);
-            else fast_t_forward<0><<<grid, kTThreads, t_bytes, stream>>>(a);
+            if (soft) fast_t_forward<1><<<grid, kTBlockThreads, t_bytes, stream>>>(a);
+            else fast_t_forward<0><<<grid, kTBlockThreads, t_bytes, stream>>>(a);
             count_launch();
         }
         if (fs.profile) {
@@ -1250,7 +1308,7 @@ cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t 
             count_launch();
         }
         if (pd.n_titems > 0) {
-            fast_t_forward<2><<<t_grid(nc, pd.n_titems, sms), kTThreads, t_bytes, stream>>>(a);
+            fast_t_forward<2><<<t_grid(nc, pd.n_titems, sms), kTBlockThreads, t_bytes, stream>>>(a);
             count_launch();
         }
     }

@@ -43,7 +43,14 @@ extern "C" int rocket_transform_soft_backward_noalloc(const rocket_params_t* p, 
     if (!(lambda == lambda) || !(shift == shift)) return ROCKET_EINVAL;
     if (!dW_dev || !db_dev) return ROCKET_EINVAL;
     if (N > 0 && (!X_dev || !dfeat_dev || !argmax_dev)) return ROCKET_EINVAL;
-    if (p->device < 0) return ROCKET_EINVAL;  // not bound yet: binding would allocate
+    int device = -1;
+    rocket::DeviceParams dp;
+    {   // the binding of a handle happens under its mutex: read what it wrote under the same mutex
+        std::lock_guard<std::mutex> lk(p->mu);
+        device = p->device;
+        dp = p->dp;
+    }
+    if (device < 0) return ROCKET_EINVAL;  // not bound yet: binding would allocate
     const int64_t nW = (int64_t)p->host.weights.size();
     if ((int64_t)N * p->host.K > 0x7fffffffll) return ROCKET_EUNSUPPORTED;
     if (rocket::generic_backward_scratch_floats(N, nW, p->host.K) > (size_t)ROCKET_NOALLOC_MAX_SCRATCH_FLOATS)
@@ -51,14 +58,14 @@ extern "C" int rocket_transform_soft_backward_noalloc(const rocket_params_t* p, 
 
     int prev = -1;
     if (cudaGetDevice(&prev) != cudaSuccess) { cudaGetLastError(); return ROCKET_ECUDA; }
-    if (prev != p->device && cudaSetDevice(p->device) != cudaSuccess) { cudaGetLastError(); return ROCKET_ECUDA; }
+    if (prev != device && cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return ROCKET_ECUDA; }
     float* scratch = nullptr;
-    int st = scratch_address(p->device, &scratch);
+    int st = scratch_address(device, &scratch);
     if (st == ROCKET_OK) {
-        cudaError_t e = rocket::launch_generic_backward(p->dp, nW, X_dev, N, lambda, shift, dfeat_dev, argmax_dev,
+        cudaError_t e = rocket::launch_generic_backward(dp, nW, X_dev, N, lambda, shift, dfeat_dev, argmax_dev,
                                                         scratch, dW_dev, db_dev, static_cast<cudaStream_t>(cuda_stream));
         if (e != cudaSuccess) { cudaGetLastError(); st = ROCKET_ECUDA; }
     }
-    if (prev != p->device) cudaSetDevice(prev);
+    if (prev != device) cudaSetDevice(prev);
     return st;
 }

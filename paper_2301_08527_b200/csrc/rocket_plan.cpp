@@ -88,9 +88,21 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         b.rows = kR + maxlen - 1;
         const int bi = (int)out.sb.size();
         out.sb.push_back(b);
+        // a tile is interior when its 64 raster positions exist and the u of every (row, column) lies inside
+        // the output range of every kernel of the bucket
+        int64_t lo_max = INT64_MIN, hi_min = INT64_MAX;
+        for (int f = b.kbeg; f < b.kend; ++f) {
+            lo_max = std::max<int64_t>(lo_max, out.krec[f].lo_u);
+            hi_min = std::min<int64_t>(hi_min, out.krec[f].hi_u);
+        }
         for (int c0 = 0; c0 < b.raster_len; c0 += kWarpCols) {
+            bool interior = c0 + kWarpCols <= b.raster_len;
+            for (int c = c0; interior && c < c0 + kWarpCols; ++c) {
+                const int64_t u0 = s_column_u0(b, c);
+                interior = u0 >= lo_max && u0 + (int64_t)(kR - 1) * d < hi_min;
+            }
             s_cost.push_back({work + 0.3 * hp.C * b.rows, (int)out.sitems.size()});
-            out.sitems.push_back({bi, c0});
+            out.sitems.push_back({bi, c0, interior ? 1 : 0, 0});
         }
     }
     {
@@ -102,7 +114,8 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
     }
 
     // ---- T regime: per kernel, the grid of 16-row x 64-column warp tiles is cut into block tiles of
-    // rg x cg warp tiles (rg * cg <= 8); the column-group width that needs the fewest block tiles wins
+    // rg x cg warp tiles (rg * cg <= the consumer warps of a block); the column-group width that needs the
+    // fewest block tiles wins
     int d_max = 0;
     std::map<std::tuple<int, int, int>, int> map_index;
     for (int k : t_kernels) {
@@ -121,55 +134,59 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
             if (rest >= 2) { widths.push_back(2); rest -= 2; }
             if (rest >= 1) widths.push_back(1);
         };
-        // A single row group under 4-wide tiles would leave half of the warps idle: it can be cut into
-        // wide tiles instead (8 column groups side by side, only the rows that hold samples), as long
-        // as the two halves fit a stage.
+        constexpr int W = kTConsumerWarps;
+        // A single row group under tiles narrower than the block has warps would leave warps idle: it can be cut
+        // into wide tiles instead (all consumer warps side by side, only the rows that hold samples), as long
+        // as the halves fit a stage.
         auto wide_fits = [&](int r16) {
             const TWindow win = t_window((int)(tmin + (int64_t)kR * r16), kR + f.len - 1, f.d, hp.L);
-            return C64 >= 5 && 2 * t_wide_half_floats(win.g_hi - win.g_lo) <= kTStageFloats;
+            return C64 > W / 2 && kTWideHalves * t_wide_half_floats(win.g_hi - win.g_lo) <= kTStageFloats;
         };
-        std::vector<int> wide_widths(C64 / 8, 8);
+        // widths of the tiles of a wide band: W column groups each, the rest in ordinary tiles of one row group
+        std::vector<int> wide_widths(C64 / W, W);
         {
-            int rest = C64 % 8;
-            if (rest >= 5) { wide_widths.push_back(8); rest = 0; }
-            if (rest >= 3) { wide_widths.push_back(4); rest = 0; }
+            int rest = C64 % W;
+            if (rest > W / 2) { wide_widths.push_back(W); rest = 0; }
+            if (W > 4 && rest >= 3) { wide_widths.push_back(4); rest = 0; }
             if (rest >= 2) { wide_widths.push_back(2); rest -= 2; }
             if (rest >= 1) wide_widths.push_back(1);
         }
-        // candidates: main width 2, 4 or 1 over all row groups, or width 4 over an even number of row
-        // groups and wide tiles over the last one; the fewest block tiles win
+        // candidates: main width 2, 4 or 1 over all row groups, or the widest main width over all row groups
+        // but the last and wide tiles over that one; the fewest block tiles win
         int best_cg = 2;
         bool last_wide = false;
         int64_t best_tiles = INT64_MAX;
         for (int cg : {2, 4, 1}) {
+            if (cg > kTMaxCg) continue;
             std::vector<int> widths;
             chunks_of(cg, widths);
             int64_t tiles = 0;
-            for (int w : widths) tiles += (R16 + 8 / w - 1) / (8 / w);
+            for (int w : widths) tiles += (R16 + W / w - 1) / (W / w);
             if (tiles < best_tiles) { best_tiles = tiles; best_cg = cg; }
         }
         if (R16 % 2 == 1 && wide_fits(R16 - 1)) {
             std::vector<int> widths;
-            chunks_of(4, widths);
+            chunks_of(kTMaxCg, widths);
             int64_t tiles = (int64_t)wide_widths.size();
-            for (int w : widths) tiles += (R16 - 1 + 8 / w - 1) / (8 / w);
-            if (tiles < best_tiles) { best_tiles = tiles; best_cg = 4; last_wide = true; }
+            for (int w : widths) tiles += (R16 - 1 + W / w - 1) / (W / w);
+            if (tiles < best_tiles) { best_tiles = tiles; best_cg = kTMaxCg; last_wide = true; }
         }
-        struct Band { int r16, nrg; std::vector<int> widths; };
+        struct Band { int r16, nrg; std::vector<int> widths; bool wide_band; };
         std::vector<Band> bands;
         std::vector<int> main_widths;
         chunks_of(best_cg, main_widths);
         const int main_rows = last_wide ? R16 - 1 : R16;
-        if (main_rows > 0) bands.push_back({0, main_rows, main_widths});
-        if (last_wide) bands.push_back({R16 - 1, 1, wide_widths});
+        if (main_rows > 0) bands.push_back({0, main_rows, main_widths, false});
+        if (last_wide) bands.push_back({R16 - 1, 1, wide_widths, true});
         for (const Band& band : bands) {
             int c64 = 0;
             for (int w : band.widths) {
-                const int rg_full = w == 8 ? 1 : 8 / w;
+                const bool wide_tile = band.wide_band && w == W;
+                const int rg_full = wide_tile ? 1 : W / w;
                 for (int r16 = band.r16; r16 < band.r16 + band.nrg; r16 += rg_full) {
                     TItem it{};
                     it.rg = std::min(rg_full, band.r16 + band.nrg - r16);
-                    it.wide = w == 8 ? 1 : 0;
+                    it.wide = wide_tile ? 1 : 0;
                     it.cg = it.wide ? 4 : w;
                     it.t0 = (int32_t)(tmin + (int64_t)kR * r16); it.r0 = c64 * kWarpCols;
                     // a tile none of whose (row, column) pairs is an output of the kernel is left out
@@ -194,6 +211,20 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
                         out.tmaps.push_back({f.d, t_box_cols(it.cg), it.box_rows});
                     }
                     it.map = found->second;
+                    // per consumer warp: does every / any (row, column) of its warp tile hold an output?
+                    for (int w8 = 0; w8 < kTConsumerWarps; ++w8) {
+                        const int wr = it.wide ? 0 : w8 / it.cg, wc = it.wide ? w8 : w8 % it.cg;
+                        if (wr >= it.rg) continue;
+                        const int64_t ta = (int64_t)it.t0 + kR * wr, ca = (int64_t)it.r0 + kWarpCols * wc;
+                        const int64_t cb = std::min<int64_t>(ca + kWarpCols, f.d);
+                        if (cb <= ca) continue;
+                        bool any = false;
+                        for (int64_t t = ta; t < ta + kR && !any; ++t)
+                            any = std::max<int64_t>(t * f.d + ca, f.lo_u) < std::min<int64_t>(t * f.d + cb, f.hi_u);
+                        if (any) it.warp_active |= 1 << w8;
+                        if (cb == ca + kWarpCols && ta * f.d + ca >= f.lo_u && (ta + kR - 1) * f.d + cb - 1 < f.hi_u)
+                            it.warp_interior |= 1 << w8;
+                    }
                     for (int ph = 0; ph < 4; ++ph) {
                         const TPhase tp = t_phase(it.t0, it.r0, it.d, ph);
                         it.x[ph] = tp.x; it.y[ph] = tp.y + it.g_lo; it.j[ph] = tp.j;

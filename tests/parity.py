@@ -1,8 +1,12 @@
 """Shared comparison rules for the GPU-vs-oracle parity tests (tolerances written out here).
 
-  max          |gpu - oracle| <= 1e-5 * max(|oracle|, 1)   (inputs are z-normalised and biases lie
-               in [-1, 1), so 1 is the scale of the summed terms; a purely relative test would
-               reject correctly rounded fp32 sums whose value happens to fall near zero)
+  max          |gpu - oracle| <= 1e-5 * max(|oracle|, 1): the stated bound, relative error <= 1e-5,
+               wherever |oracle| >= 1, and the same bound with |oracle| replaced by 1 below that
+               (inputs are z-normalised and biases lie in [-1, 1), so 1 is the scale of the summed
+               terms; a purely relative test would reject correctly rounded fp32 sums whose value
+               happens to fall near zero: a sum of 30-120 products of size ~1 carries an fp32
+               rounding error of a few 1e-7 whatever its own size).  check_max returns the share of
+               pairs under the floor and the worst purely relative error on both sides of it.
   hard PPV     count accepted iff  P+ - 1e-4 n <= count <= P+ + AMB + 1e-4 n,  where P+ counts
                oracle outputs above 1e-5 and AMB those within 1e-5 of zero (their sign is not
                decidable in fp32)
@@ -21,11 +25,23 @@ GRAD_REL_L2 = 1e-4
 
 
 def check_max(gpu_max, ref):
+    """Asserts the max rule; returns a dict with the worst scaled error, the share of pairs whose
+    |oracle max| lies under the floor of 1, and the worst purely relative error at or above / below
+    the floor (the latter is reported, not asserted)."""
     gpu_max = np.asarray(gpu_max, np.float64)
-    err = np.abs(gpu_max - ref.max) / np.maximum(np.abs(ref.max), 1.0)
+    ref_max = np.asarray(ref.max, np.float64)
     assert np.all(np.isfinite(gpu_max))
-    assert err.max(initial=0.0) <= MAX_RTOL, "max rel err %.3g at %s" % (err.max(), np.argmax(err))
-    return float(err.max(initial=0.0))
+    diff = np.abs(gpu_max - ref_max)
+    err = diff / np.maximum(np.abs(ref_max), 1.0)
+    assert err.max(initial=0.0) <= MAX_RTOL, "max err %.3g (scaled) at %s" % (err.max(), np.argmax(err))
+    big = np.abs(ref_max) >= 1.0
+    with np.errstate(divide="ignore", invalid="ignore"):
+        rel = np.where(ref_max != 0.0, diff / np.abs(ref_max), np.where(diff == 0.0, 0.0, np.inf))
+    rel_big = float(rel[big].max(initial=0.0))
+    assert rel_big <= MAX_RTOL, "max relative err %.3g where |max| >= 1" % rel_big
+    return {"scaled_err": float(err.max(initial=0.0)), "share_below_floor": float(1.0 - big.mean()) if big.size else 0.0,
+            "rel_err_at_or_above_floor": rel_big, "rel_err_below_floor": float(rel[~big].max(initial=0.0)),
+            "share_below_floor_over_1e-5": float((rel[~big] > MAX_RTOL).sum() / big.size) if big.size else 0.0}
 
 
 def check_hard_ppv(gpu_ppv, ref):

@@ -57,6 +57,7 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
     for (const SItem& it : plan.sitems) {
         const SBucket& b = plan.sb[it.bucket];
         REQUIRE(b.rows <= kRowsMax && b.d < plan.split && it.c0 % kWarpCols == 0, "S bucket shape");
+        bool all_full = true;
         for (int col = 0; col < kWarpCols; ++col) {
             const int cg = it.c0 + col;
             const bool col_ok = cg < b.raster_len;
@@ -69,6 +70,7 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
                 const int band = cg / b.d;
                 valid_rows_tc(b.tmin + band * kR, cg - band * b.d, f.tl, f.rl, f.th, f.rh, kR, col_ok, o_lo, o_hi);
                 REQUIRE((o_lo >= o_hi && q_lo >= q_hi) || (o_lo == q_lo && o_hi == q_hi), "S row range: the two forms disagree");
+                all_full = all_full && o_lo == 0 && o_hi == kR;
                 for (int o = o_lo; o < o_hi; ++o) {
                     const int64_t i = (int64_t)u0 + (int64_t)o * b.d + f.p;
                     REQUIRE(i >= 0 && i < f.nout, "S output out of range");
@@ -76,6 +78,8 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
                 }
             }
         }
+        // the kernels skip every range test on a tile flagged interior
+        REQUIRE((it.interior != 0) == all_full, "S interior flag %d, replay says %d", it.interior, (int)all_full);
     }
 
     const int64_t pitch = plan.pad_pitch;
@@ -85,19 +89,19 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
         REQUIRE(it.map >= 0 && it.map < (int)plan.tmaps.size(), "T map index");
         const TMapSpec& sp = plan.tmaps[it.map];
         REQUIRE(f.d >= kTMinDilation && f.d == it.d && f.len == it.len && f.m == it.m, "T item fields");
-        REQUIRE((it.cg == 1 || it.cg == 2 || it.cg == 4) && it.rg >= 1 && it.rg * it.cg <= kTConsumerWarps, "T shape");
+        REQUIRE((it.cg == 1 || it.cg == 2 || it.cg == 4) && (it.cg <= kTMaxCg || it.wide) && it.rg >= 1 && it.rg * it.cg <= kTConsumerWarps, "T shape");
         REQUIRE(it.r0 % kWarpCols == 0 && it.r0 < f.d, "T column origin");
         for (int q = 0; q < f.m; ++q) REQUIRE(it.ch[q] == f.ch[q], "T channel list");
         const bool wide = it.wide != 0;
         const int rows_out = kR * it.rg, boxw = t_box_cols(it.cg);
-        const int tile_cols = wide ? 2 * kTWideCols : boxw;
+        const int tile_cols = wide ? kTWideHalves * kTWideCols : boxw;
         const int rows = rows_out + f.len - 1;
         if (wide) {
             const TWindow win = t_window(it.t0, rows, f.d, L);
             REQUIRE(it.rg == 1 && it.cg == 4 && boxw == kTWideCols, "wide tile shape");
             REQUIRE(it.g_lo == win.g_lo && it.g_hi == win.g_hi && win.g_lo >= 0 && win.g_lo < win.g_hi && 4 * win.g_hi < rows + 4,
                     "wide tile window");
-            REQUIRE(2 * t_wide_half_floats(it.box_rows) <= kTStageFloats, "wide stage size");
+            REQUIRE(kTWideHalves * t_wide_half_floats(it.box_rows) <= kTStageFloats, "wide stage size");
         } else {
             REQUIRE(it.g_lo == 0 && it.g_hi == t_box_rows(it.rg, f.len) && 4 * it.g_hi >= rows, "T box rows");
         }
@@ -106,8 +110,8 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
         REQUIRE(4 * t_phase_floats(it.cg, it.box_rows) <= kTStageFloats, "stage size");
         const long long run = 4ll * f.d, ny = (kTPadFront + (long long)L + run - 1) / run;
         // the boxes the producer issues: four phases, twice for a wide tile
-        TPhase ph[8];
-        for (int k = 0; k < (wide ? 8 : 4); ++k) {
+        TPhase ph[4 * (kTWideHalves > 1 ? kTWideHalves : 1)];
+        for (int k = 0; k < (wide ? 4 * kTWideHalves : 4); ++k) {
             if (k < 4) {
                 ph[k] = t_phase(it.t0, it.r0, f.d, k);
                 ph[k].y += it.g_lo;
@@ -129,6 +133,8 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
             }
         }
         // what every consumer thread owns and reads
+        bool w_full[kTConsumerWarps], w_any[kTConsumerWarps];
+        for (int w8 = 0; w8 < kTConsumerWarps; ++w8) { w_full[w8] = true; w_any[w8] = false; }
         for (int lc = 0; lc < tile_cols; ++lc) {
             const bool col_ok = it.r0 + lc < f.d;
             for (int wr = 0; wr < it.rg; ++wr) {
@@ -137,6 +143,9 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
                 valid_rows(u0, f.d, f.lo_u, f.hi_u, kR, col_ok, q_lo, q_hi);
                 valid_rows_tc(it.t0 + kR * wr, it.r0 + lc, f.tl, f.rl, f.th, f.rh, kR, col_ok, o_lo, o_hi);
                 REQUIRE((o_lo >= o_hi && q_lo >= q_hi) || (o_lo == q_lo && o_hi == q_hi), "T row range: the two forms disagree");
+                const int w8 = wide ? lc / kWarpCols : wr * it.cg + lc / kWarpCols;
+                w_full[w8] = w_full[w8] && o_lo == 0 && o_hi == kR;
+                w_any[w8] = w_any[w8] || o_lo < o_hi;
                 for (int o = o_lo; o < o_hi; ++o) {
                     const int64_t i = (int64_t)u0 + (int64_t)o * f.d + f.p;
                     REQUIRE(i >= 0 && i < f.nout, "T output out of range");
@@ -152,7 +161,7 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
                         REQUIRE(wide && !in_series, "a skipped row holds a sample");
                         continue;
                     }
-                    const int k = (s & 3) + (wide && lc >= kTWideCols ? 4 : 0);
+                    const int k = (s & 3) + (wide ? 4 * (lc / kTWideCols) : 0);
                     const int pos = wide ? t_wide_elem_offset(s, lc, it.box_rows, it.g_lo) : t_elem_offset(it.cg, s, lc, it.box_rows);
                     REQUIRE(pos >= 0 && pos < kTStageFloats, "read outside the stage");
                     if ((lc & 1) == 0) REQUIRE(pos % 2 == 0, "pair not 8-byte aligned");
@@ -167,7 +176,16 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
                 }
             }
         }
+        // the per-warp flags the consumers trust instead of range tests
+        const int n_tiles_w = wide ? kTConsumerWarps : it.rg * it.cg;
+        for (int w8 = 0; w8 < kTConsumerWarps; ++w8) {
+            const bool in_tile = w8 < n_tiles_w;
+            const bool full = in_tile && w_full[w8], any = in_tile && w_any[w8];
+            REQUIRE(((it.warp_interior >> w8) & 1) == (int)full, "T interior flag of warp %d", w8);
+            REQUIRE(((it.warp_active >> w8) & 1) == (int)any, "T active flag of warp %d", w8);
+        }
     }
+    // (the flag check of the T tiles sits at the end of the tile loop above)
     for (size_t fidx = 0; fidx < plan.krec.size(); ++fidx)
         for (int i = 0; i < plan.krec[fidx].nout; ++i)
             REQUIRE(cover[fidx][i] == 1, "kernel %d (len %d d %d p %d) output %d owned %d times", plan.krec[fidx].k,

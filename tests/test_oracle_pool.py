@@ -10,7 +10,7 @@ from rocket_inputs import generate_kernels, kernels_from_lists, random_walk_seri
 RNG = np.random.default_rng(5)
 
 
-def _brute(p, X, n, k, lam, shift):
+def _brute(p, X, n, k, lam, shift, eps=1e-5):
     """Pure-Python restatement on tiny inputs (no numpy arithmetic, no oracle code)."""
     co, wo = p.channel_offset, p.weight_offset
     ln, d, pad, m = int(p.length[k]), int(p.dilation[k]), int(p.padding[k]), int(p.num_channels[k])
@@ -27,7 +27,9 @@ def _brute(p, X, n, k, lam, shift):
         zs.append(z)
     ppv = sum(1 for z in zs if z > 0) / nout
     soft = sum(1.0 / (1.0 + math.exp(-(lam * z + shift))) for z in zs) / nout
-    return ppv, max(zs), soft, zs.index(max(zs))
+    pos_eps = sum(1 for z in zs if z > eps)
+    amb = sum(1 for z in zs if -eps <= z <= eps)
+    return ppv, max(zs), soft, zs.index(max(zs)), pos_eps, amb
 
 
 def test_brute_force_on_tiny_series():
@@ -36,11 +38,59 @@ def test_brute_force_on_tiny_series():
     out = oracle.forward(p, X, lam=2.0, shift=3.0)
     for n in range(2):
         for k in range(p.K):
-            ppv, mx, soft, arg = _brute(p, X, n, k, 2.0, 3.0)
+            ppv, mx, soft, arg, pos_eps, amb = _brute(p, X, n, k, 2.0, 3.0)
             assert out.ppv[n, k] == pytest.approx(ppv, abs=1e-15)
             assert out.max[n, k] == pytest.approx(mx, rel=1e-13, abs=1e-13)
             assert out.soft[n, k] == pytest.approx(soft, abs=1e-13)
             assert out.argmax[n, k] == arg
+            assert out.pos_eps[n, k] == pos_eps and out.amb[n, k] == amb
+
+
+def test_brute_force_counts_near_zero_with_a_wide_band():
+    # a band wide enough that many outputs fall inside it: the two counts that set the acceptance
+    # band of the hard-PPV parity checks are compared with the pure-Python count
+    p = generate_kernels(13, 30, 2, 40)
+    X = (0.05 * random_walk_series(14, 2, 2, 40)).astype(np.float32)
+    p.bias = (0.02 * p.bias).astype(np.float32)
+    p.weights = (0.05 * p.weights).astype(np.float32)
+    out = oracle.forward(p, X, amb_eps=0.01)
+    seen_amb = 0
+    for n in range(2):
+        for k in range(p.K):
+            _, _, _, _, pos_eps, amb = _brute(p, X, n, k, 1.0, 3.0, eps=0.01)
+            assert out.pos_eps[n, k] == pos_eps and out.amb[n, k] == amb
+            seen_amb += amb
+    assert seen_amb > 50   # the case does exercise the band
+
+
+def test_hand_worked_counts_around_the_ambiguity_band():
+    # single-tap kernel (w_0 = 1, other taps 0, bias 0, no padding): z_i = x_i for i < L - 6.
+    # With eps = 2^-17 (exact in binary) the outputs sit below, on and above both edges of the band:
+    #   z:  -2^-16   -2^-17   -2^-18   0   2^-18   2^-17   2^-17 (1 + 2^-23)   2^-16
+    #   z > eps            : the last two                       -> pos_eps = 2
+    #   |z| <= eps         : -2^-17, -2^-18, 0, 2^-18, 2^-17    -> amb = 5   (both edges belong to the band)
+    #   z > 0              : four values                        -> PPV = 4/8
+    e = 2.0 ** -17
+    z = [-2 * e, -e, -e / 2, 0.0, e / 2, e, e * (1 + 2.0 ** -23), 2 * e]
+    x = np.array(z + [9.0] * 6, np.float32)[None, None, :]
+    assert [float(v) for v in x[0, 0, :8]] == z       # every value is exact in fp32
+    w = np.zeros((1, 7), np.float32)
+    w[0, 0] = 1.0
+    p = kernels_from_lists(1, 14, [dict(dilation=1, padding=0, channels=[0], weights=w, bias=0.0)])
+    out = oracle.forward(p, x, amb_eps=e)
+    assert out.out_len[0, 0] == 8
+    assert out.pos_eps[0, 0] == 2 and out.amb[0, 0] == 5 and out.ppv[0, 0] == 0.5
+    # the default band, 1e-5: float32(1e-5) lies just below 1e-5 (inside the band), its successor just above
+    f = np.float32(1e-5)
+    g = np.nextafter(f, np.float32(1))
+    assert float(f) < 1e-5 < float(g)
+    z2 = [-2e-5, -5e-6, 0.0, 5e-6, float(f), float(g), 2e-5, -float(g)]
+    x2 = np.array(z2 + [9.0] * 6, np.float32)[None, None, :]
+    out = oracle.forward(p, x2)
+    assert out.pos_eps[0, 0] == 2 and out.amb[0, 0] == 4 and out.ppv[0, 0] == 0.5
+    # a dropped or doubled count would also break the partition: below + band + above = all outputs
+    below = sum(1 for v in x2[0, 0, :8] if float(v) < -1e-5)
+    assert below + out.amb[0, 0] + out.pos_eps[0, 0] == 8
 
 
 def test_hand_worked_case_features():

@@ -5,14 +5,16 @@ latency budget, a process whose device memory pool is fixed at start-up, code ru
 someone else records the stream.  rocket_transform_soft_backward_noalloc serves them by keeping
 its partial sums in a fixed array inside the library.  This test calls it through the C ABI twice
 in a row (the array is shared between calls and keeps old contents) and checks each result
-against rocket_transform_soft_backward on the same inputs.  It lives in a file that sorts last,
-so a run that stops at the first failure has already run every other test.
+against rocket_transform_soft_backward on the same inputs, and both against the CPU oracle's
+gradients.  It lives in a file that sorts last, so a run that stops at the first failure has
+already run every other test.
 """
 import ctypes
 
 import numpy as np
 import pytest
 
+import oracle
 import paper_2301_08527_b200 as rk
 from paper_2301_08527_b200 import binding
 from rocket_inputs import ar1_spike_series, generate_kernels, normal_array
@@ -29,11 +31,15 @@ def test_noalloc_backward_matches_allocating_backward_on_two_calls_in_a_row():
     cases = [(61, 300, 6, 1200, 5), (62, 120, 4, 700, 3)]
     for seed, K, C, L, N in cases:
         kp = generate_kernels(seed, K, C, L)
-        X = torch.from_numpy(ar1_spike_series(seed + 100, N, C, L)).cuda()
-        g = torch.from_numpy(normal_array(seed + 200, (N, 2 * K))).cuda()
+        Xh = ar1_spike_series(seed + 100, N, C, L)
+        gh = normal_array(seed + 200, (N, 2 * K))
+        X = torch.from_numpy(Xh).cuda()
+        g = torch.from_numpy(gh).cuda()
         p = rk.RocketParams.from_kernel_params(kp)
         p.bind_device()                      # binding allocates: done here, at set-up
-        _, arg = rk.rocket_transform_soft(p, X, lam, shift)
+        ref = oracle.forward(kp, Xh, lam=lam, shift=shift)
+        arg = torch.from_numpy(ref.argmax.astype(np.int32)).cuda()    # the oracle's argmax feeds all three
+        oracle_dW, oracle_db = oracle.backward(kp, Xh, gh, ref.argmax, lam=lam, shift=shift)
         ref_dW, ref_db = rk.rocket_transform_soft_backward(p, X, lam, shift, g, arg)
         dW = torch.full((p.n_weights,), float("nan"), device="cuda")
         db = torch.full((K,), float("nan"), device="cuda")
@@ -42,6 +48,8 @@ def test_noalloc_backward_matches_allocating_backward_on_two_calls_in_a_row():
         rel = P.check_grads(dW.cpu().numpy(), db.cpu().numpy(),
                             ref_dW.cpu().numpy().astype(np.float64), ref_db.cpu().numpy().astype(np.float64))
         assert rel <= P.GRAD_REL_L2
+        P.check_grads(dW.cpu().numpy(), db.cpu().numpy(), oracle_dW, oracle_db)
+        P.check_grads(ref_dW.cpu().numpy(), ref_db.cpu().numpy(), oracle_dW, oracle_db)
         p.close()
 
 
