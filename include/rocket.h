@@ -23,10 +23,18 @@
  *   - Kernel parameters are ragged: kernel k owns num_channels[k] consecutive entries of
  *     channel_idx and num_channels[k]*length[k] consecutive weights, row-major [q][j].
  *   - Device calls enqueue work on the caller's stream (a cudaStream_t passed as void*, NULL =
- *     the legacy default stream) and return without synchronising.  Outputs are fully
- *     overwritten.  The caller owns every buffer it passes; the library owns the handle and
- *     the workspace inside it.  Two calls that use the same handle must be ordered on the
- *     device (same stream, or an event between them): they share the handle's workspace.
+ *     the legacy default stream).  Outputs are fully overwritten.  The caller owns every buffer
+ *     it passes; the library owns the handle and the workspace inside it.  Two calls that use
+ *     the same handle must be ordered on the device (same stream, or an event between them):
+ *     they share the handle's workspace.
+ *   - Workspace.  The handle's workspace (parameter upload, zero-margined staging copies and
+ *     their tensor maps, per-pair and per-weight accumulators) is allocated either up front by
+ *     rocket_params_reserve, or lazily: the first device call, the first call of a kind (soft,
+ *     backward, 8-bit input) and any call with more examples than every call before it may
+ *     allocate, free, clear and upload, which synchronises the device.  Once the workspace
+ *     covers a call - after rocket_params_reserve for its size and passes, or after an earlier
+ *     call at least as large - the device calls only enqueue kernels and return without
+ *     allocating or synchronising.  rocket_device_alloc_count lets a caller verify that.
  *   - Every function returns a rocket_status_t (0 = success).  Argument errors are detected
  *     on the host before anything is launched and leave the outputs untouched.  Nothing
  *     aborts and nothing throws across this boundary.  There is no CPU fallback: without a
@@ -106,6 +114,27 @@ int rocket_params_work(const rocket_params_t* p, double* conv_flops_per_example,
  * first device call.  Allocates device memory; a no-op returning ROCKET_OK when already bound.
  */
 int rocket_params_bind_device(const rocket_params_t* p);
+
+/*
+ * Allocate, now, everything the device calls with this handle will need for up to max_N examples
+ * per call, on the current device (binding the handle to it if it is not bound yet), so that the
+ * calls themselves never allocate, free or synchronise.  passes is a bit set of the calls to
+ * prepare for: ROCKET_PASS_HARD (rocket_transform), ROCKET_PASS_SOFT (rocket_transform_soft),
+ * ROCKET_PASS_BACKWARD (rocket_transform_soft_backward) and ROCKET_PASS_U8_INPUT (the *_u8 forms of
+ * the passes named).  May be called again with a larger max_N or more passes; never shrinks.  The
+ * host-buffer forms (*_host) stage through buffers of their own and synchronise by design; they
+ * are not covered.  ROCKET_EINVAL for max_N < 1 or an empty / unknown set of passes, ROCKET_ENOMEM
+ * when the device memory does not suffice (what was allocated before stays usable).
+ */
+#define ROCKET_PASS_HARD 1
+#define ROCKET_PASS_SOFT 2
+#define ROCKET_PASS_BACKWARD 4
+#define ROCKET_PASS_U8_INPUT 8
+int rocket_params_reserve(rocket_params_t* p, int max_N, int passes);
+
+/* Number of device allocations (cudaMalloc) the library has made in this process so far.  A
+ * caller that must not allocate in its steady state reads it before and after a call. */
+int64_t rocket_device_alloc_count(void);
 
 /* Free the handle, its device copies and its workspace.  NULL is allowed.  The caller must
  * have synchronised any stream that still runs work enqueued with this handle. */

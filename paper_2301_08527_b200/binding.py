@@ -38,6 +38,8 @@ SIGNATURES = {
                                                               ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p,
                                                               ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "rocket_kernel_launch_count": (ctypes.c_int64, []),
+    "rocket_device_alloc_count": (ctypes.c_int64, []),
+    "rocket_params_reserve": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_int]),
     "rocket_params_set_profiling": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
     "rocket_params_last_profile": (ctypes.c_int, [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_double)] * 4),
     "rocket_transform": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
@@ -101,6 +103,13 @@ def load_library():
 def _check(status, where):
     if status != 0:
         raise RocketError(status, where)
+
+
+PASS_HARD, PASS_SOFT, PASS_BACKWARD, PASS_U8_INPUT = 1, 2, 4, 8
+
+
+def device_alloc_count():
+    return int(load_library().rocket_device_alloc_count())
 
 
 def kernel_launch_count():
@@ -170,6 +179,10 @@ class RocketParams:
     def bind_device(self):
         """rocket_params_bind_device: upload the parameters to the current device now."""
         _check(load_library().rocket_params_bind_device(self._h), "rocket_params_bind_device")
+
+    def reserve(self, max_N, passes=PASS_HARD):
+        _check(load_library().rocket_params_reserve(self._h, ctypes.c_int(int(max_N)), ctypes.c_int(int(passes))),
+               "rocket_params_reserve")
 
     def device_status(self):
         """rocket_params_device_status: number of bounded waits that gave up (0 = healthy)."""

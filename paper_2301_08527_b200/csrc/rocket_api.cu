@@ -9,6 +9,7 @@
 
 namespace rocket {
 std::atomic<int64_t> g_launch_count{0};
+std::atomic<int64_t> g_alloc_count{0};
 }
 
 using namespace rocket;
@@ -73,7 +74,7 @@ int ensure_device(const rocket_params* p) {
         {h.bias.data(), h.bias.size() * 4, 0}};
     size_t total = 0;
     for (auto& pt : parts) { pt.off = total; total += align256(pt.bytes); }
-    cudaError_t e = cudaMalloc(&p->dev_blob, std::max<size_t>(total, 256));
+    cudaError_t e = device_malloc(&p->dev_blob, std::max<size_t>(total, 256));
     if (e != cudaSuccess) { cudaGetLastError(); p->dev_blob = nullptr; return e == cudaErrorMemoryAllocation ? ROCKET_ENOMEM : ROCKET_ECUDA; }
     char* base = static_cast<char*>(p->dev_blob);
     for (auto& pt : parts)
@@ -341,6 +342,37 @@ int rocket_params_last_profile(const rocket_params_t* p, double* ms_small_dilati
 }
 
 int64_t rocket_kernel_launch_count(void) { return g_launch_count.load(std::memory_order_relaxed); }
+
+int64_t rocket_device_alloc_count(void) { return g_alloc_count.load(std::memory_order_relaxed); }
+
+int rocket_params_reserve(rocket_params_t* p, int max_N, int passes) {
+    if (!p || max_N < 1 || passes < 1 || passes > 15) return ROCKET_EINVAL;
+    if ((int64_t)max_N * p->host.K > 0x7fffffffll) return ROCKET_EUNSUPPORTED;
+    int st = ensure_device(p);
+    if (st != ROCKET_OK) return st;
+    DeviceGuard g(p->device);
+    if (!g.ok) return ROCKET_ECUDA;
+    const bool soft = (passes & ROCKET_PASS_SOFT) != 0, backward = (passes & ROCKET_PASS_BACKWARD) != 0;
+    const bool u8 = (passes & ROCKET_PASS_U8_INPUT) != 0;
+    const int64_t nW = n_weights_of(p);
+    if (p->fast->host.enabled) {
+        cudaError_t e = fast::reserve_fast_state(*p->fast, p->dp, max_N, soft, backward, u8, nW);
+        if (e != cudaSuccess) return cuda_status(e);
+    }
+    std::lock_guard<std::mutex> lk(p->mu);
+    // kernels outside the fused path: the backward's per-example partial sums; 8-bit input: its fp32 copy
+    const bool some_generic = !p->fast->host.enabled || !p->fast->host.generic_list.empty() || p->path == 1;
+    if (backward && some_generic) {
+        cudaError_t e = p->scratch.reserve(generic_backward_scratch_floats(max_N, nW, p->host.K) * sizeof(float));
+        if (e != cudaSuccess) return cuda_status(e);
+    }
+    if (u8 && (some_generic || p->host.C > fast::kNormMaxChannels)) {
+        cudaError_t e = p->u8_x.reserve((size_t)max_N * p->host.C * p->host.L * sizeof(float));
+        if (e == cudaSuccess) e = p->u8_norm.reserve((size_t)2 * p->host.C * sizeof(float));
+        if (e != cudaSuccess) return cuda_status(e);
+    }
+    return ROCKET_OK;
+}
 
 int rocket_transform(const rocket_params_t* p, const float* X_dev, int N, int C, int L, float* feat_dev,
                      void* cuda_stream) {

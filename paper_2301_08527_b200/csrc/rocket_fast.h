@@ -27,6 +27,7 @@
 #pragma once
 
 #include <cstdint>
+#include <mutex>
 #include <vector>
 
 #include "rocket_internal.h"
@@ -187,6 +188,7 @@ void build_plan(const HostParams& hp, int split, PlanHost& out);
 
 // Device-side state of the fast path owned by a handle.
 struct FastState {
+    std::mutex mu;                        // guards the grow-only buffers below and the launch sequence of a call
     PlanHost host;
     PlanDevice dev;
     void* plan_blob = nullptr;            // records, buckets, items, counters, error flag
@@ -208,6 +210,12 @@ cudaError_t upload_plan(FastState& fs);
 void release_fast_state(FastState& fs);
 // Makes the padded copy hold N examples and (re-)encodes the tensor maps over it.
 cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L, bool without_maps = false);
+
+// Allocates, once, everything the fused kernels need for calls of up to max_N examples (the zero-margined
+// copies and their tensor maps, the soft transform's and the backward's workspaces) and opts the kernels
+// into their shared-memory sizes; later calls within that size allocate nothing.
+cudaError_t reserve_fast_state(FastState& fs, const DeviceParams& dp, int max_N, bool soft, bool backward, bool u8,
+                               int64_t n_weights);
 
 // Backward of the soft transform through the fast path (every kernel must be a fast-path kernel):
 // dW (ragged like the weights, n_weights floats) and db [K] are assigned.

@@ -20,6 +20,7 @@
 #include <cfloat>
 #include <climits>
 #include <cstring>
+#include <mutex>
 
 #include "rocket_fast.h"
 #include "rocket_fast_geom.h"
@@ -973,6 +974,8 @@ EncodeTiledFn encode_tiled_fn() {
 // Opts every fused kernel into its dynamic shared memory size, once per device.
 cudaError_t set_kernel_attributes(int dev) {
     cudaError_t e = cudaSuccess;
+    static std::mutex attr_mu;
+    std::lock_guard<std::mutex> attr_lock(attr_mu);
     static bool attr_done_for[64] = {};
     bool& attr_done = attr_done_for[dev & 63];
     const size_t t_bytes = t_smem_bytes();
@@ -1059,7 +1062,7 @@ cudaError_t upload_plan(FastState& fs) {
         {h.generic_list.data(), h.generic_list.size() * 4, 0}, {nullptr, 256, 0}, {nullptr, 256, 0}};
     size_t total = 0;
     for (auto& pt : parts) { pt.off = total; total += align256(pt.bytes); }
-    cudaError_t e = cudaMalloc(&fs.plan_blob, std::max<size_t>(total, 256));
+    cudaError_t e = device_malloc(&fs.plan_blob, std::max<size_t>(total, 256));
     if (e != cudaSuccess) { fs.plan_blob = nullptr; return e; }
     char* base = static_cast<char*>(fs.plan_blob);
     e = cudaMemset(base, 0, std::max<size_t>(total, 256));
@@ -1112,7 +1115,7 @@ cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L, bool without
     if (fs.xpad) cudaFree(fs.xpad);  // waits for work that still reads it
     fs.xpad = nullptr;
     fs.pad_examples = 0;
-    cudaError_t e = cudaMalloc(&fs.xpad, bytes);
+    cudaError_t e = device_malloc(reinterpret_cast<void**>(&fs.xpad), bytes);
     if (e != cudaSuccess) { fs.xpad = nullptr; return e; }
     e = cudaMemset(fs.xpad, 0, bytes);  // the margins stay zero from here on: the pad copy writes samples only
     if (e != cudaSuccess) return e;
@@ -1133,7 +1136,7 @@ cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L, bool without
     static_assert(sizeof(CUtensorMap) == 128, "tensor maps are addressed in 128-byte steps");
     if (n_maps > 0) {
         if (!fs.maps_blob) {
-            e = cudaMalloc(&fs.maps_blob, n_maps * sizeof(CUtensorMap));
+            e = device_malloc(&fs.maps_blob, n_maps * sizeof(CUtensorMap));
             if (e != cudaSuccess) { fs.maps_blob = nullptr; return e; }
         }
         e = cudaMemcpy(fs.maps_blob, maps.data(), n_maps * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
@@ -1146,9 +1149,47 @@ cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L, bool without
     return cudaSuccess;
 }
 
+// Soft transform: 16 bytes per (example, kernel), grow-only.
+static cudaError_t ensure_soft_ws(FastState& fs, int64_t pairs) {
+    if ((size_t)pairs * 16 <= fs.soft_ws_bytes) return cudaSuccess;
+    if (fs.soft_ws) cudaFree(fs.soft_ws);  // waits for work that still uses it
+    fs.soft_ws = nullptr;
+    fs.soft_ws_bytes = 0;
+    cudaError_t e = device_malloc(&fs.soft_ws, (size_t)pairs * 16);
+    if (e != cudaSuccess) { fs.soft_ws = nullptr; return e; }
+    fs.soft_ws_bytes = (size_t)pairs * 16;
+    return cudaSuccess;
+}
+
+// Backward: fixed-point sums [n_weights + K], scales [K], max |x| (fixed size per handle).
+static cudaError_t ensure_bwd_ws(FastState& fs, const DeviceParams& dp, int64_t n_weights) {
+    if (fs.bwd_ws) return cudaSuccess;
+    const size_t acc_bytes = align256((size_t)(n_weights + dp.K) * 8), scale_bytes = align256((size_t)dp.K * 8);
+    cudaError_t e = device_malloc(&fs.bwd_ws, acc_bytes + scale_bytes + 256);
+    if (e != cudaSuccess) fs.bwd_ws = nullptr;
+    return e;
+}
+
+cudaError_t reserve_fast_state(FastState& fs, const DeviceParams& dp, int max_N, bool soft, bool backward, bool u8,
+                               int64_t n_weights) {
+    std::lock_guard<std::mutex> lk(fs.mu);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if ((e = set_kernel_attributes(dev)) != cudaSuccess) return e;
+    if (fs.dev.n_titems > 0 || u8) {
+        e = ensure_pad_capacity(fs, std::min(max_N, kChunkExamples), dp.C, dp.L, u8 && fs.dev.n_titems == 0);
+        if (e != cudaSuccess) return e;
+    }
+    if (soft && (e = ensure_soft_ws(fs, (int64_t)max_N * dp.K)) != cudaSuccess) return e;
+    if (backward && fs.host.generic_list.empty() && (e = ensure_bwd_ws(fs, dp, n_weights)) != cudaSuccess) return e;
+    return cudaSuccess;
+}
+
 cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const float* X, int N, float* feat,
                                 cudaStream_t stream, bool soft, float lambda, float shift, int32_t* argmax,
                                 const uint8_t* X_u8, const NormArgs* norm) {
+    std::lock_guard<std::mutex> lk(fs.mu);
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -1163,14 +1204,7 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
         if (e != cudaSuccess) return e;
     }
     const int64_t pairs = (int64_t)N * dp.K;
-    if (soft && (size_t)pairs * 16 > fs.soft_ws_bytes) {
-        if (fs.soft_ws) cudaFree(fs.soft_ws);  // waits for work that still uses it
-        fs.soft_ws = nullptr;
-        fs.soft_ws_bytes = 0;
-        e = cudaMalloc(&fs.soft_ws, (size_t)pairs * 16);
-        if (e != cudaSuccess) { fs.soft_ws = nullptr; return e; }
-        fs.soft_ws_bytes = (size_t)pairs * 16;
-    }
+    if (soft && (e = ensure_soft_ws(fs, pairs)) != cudaSuccess) return e;
     FwdArgs a;
     a.plan = fs.dev;
     a.c1 = lambda * 1.4426950408889634f; a.c0 = -shift * 1.4426950408889634f;
@@ -1250,6 +1284,7 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
 cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t n_weights, const float* X, int N,
                                  float lambda, float shift, const float* dfeat, const int32_t* argmax, float* dW,
                                  float* db, cudaStream_t stream) {
+    std::lock_guard<std::mutex> lk(fs.mu);
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -1261,10 +1296,7 @@ cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t 
     const PlanDevice& pd = fs.dev;
     // workspace: fixed-point sums [n_weights + K], scales [K], max |x| (fixed size per handle)
     const size_t acc_bytes = align256((size_t)(n_weights + dp.K) * 8), scale_bytes = align256((size_t)dp.K * 8);
-    if (!fs.bwd_ws) {
-        e = cudaMalloc(&fs.bwd_ws, acc_bytes + scale_bytes + 256);
-        if (e != cudaSuccess) { fs.bwd_ws = nullptr; return e; }
-    }
+    if ((e = ensure_bwd_ws(fs, dp, n_weights)) != cudaSuccess) return e;
     long long* accfix = static_cast<long long*>(fs.bwd_ws);
     double* scale = reinterpret_cast<double*>(static_cast<char*>(fs.bwd_ws) + acc_bytes);
     unsigned* absmax = reinterpret_cast<unsigned*>(static_cast<char*>(fs.bwd_ws) + acc_bytes + scale_bytes);

@@ -37,6 +37,14 @@ struct HostParams {
 extern std::atomic<int64_t> g_launch_count;
 inline void count_launch(int n = 1) { g_launch_count.fetch_add(n, std::memory_order_relaxed); }
 
+// Every device allocation of the library goes through here, so that a caller (and the tests) can
+// tell whether a call allocated: rocket_device_alloc_count reports the number made so far.
+extern std::atomic<int64_t> g_alloc_count;
+inline cudaError_t device_malloc(void** ptr, size_t bytes) {
+    g_alloc_count.fetch_add(1, std::memory_order_relaxed);
+    return cudaMalloc(ptr, bytes);
+}
+
 // Draws K kernels by the rules of Section 3.1 with the counter-based generator.
 void generate_host_params(uint64_t seed, int K, int C, int L, HostParams& out);
 
@@ -68,7 +76,7 @@ struct DeviceBuffer {
         if (need <= bytes) return cudaSuccess;
         if (ptr) cudaFree(ptr);
         ptr = nullptr; bytes = 0;
-        cudaError_t e = cudaMalloc(&ptr, need);
+        cudaError_t e = rocket::device_malloc(&ptr, need);
         if (e == cudaSuccess) bytes = need;
         else ptr = nullptr;
         return e;

@@ -203,7 +203,7 @@ extern "C" int rocket_ridge_fit(const float* feat_dev, int N, int P, const float
     // workspace: mu[P], G[N][N], a[N], part[nparts], ybar, status
     const size_t doubles = (size_t)P + (size_t)N * N + (size_t)N + (size_t)nparts + 1;
     char* ws = nullptr;
-    cudaError_t e = cudaMalloc(&ws, doubles * sizeof(double) + 16);
+    cudaError_t e = rocket::device_malloc(reinterpret_cast<void**>(&ws), doubles * sizeof(double) + 16);
     if (e != cudaSuccess) return status_of(e);
     double* mu = reinterpret_cast<double*>(ws);
     double* G = mu + P;

@@ -65,3 +65,37 @@ def test_random_geometry_all_passes(seed):
         P.check_grads(dW.cpu().numpy(), db.cpu().numpy(), rW, rb)
         assert p.device_status() == 0
         p.close()
+
+
+def test_backward_with_padding_beyond_eight_dilations_on_the_fused_kernels():
+    # paddings of 8 d to 10 d (legal for caller-supplied kernels) put outputs more than 8 rows of the dilated
+    # view before the first sample; the argmax term of the gradient must survive there.  Every kernel has a
+    # fast-path length, so the fused backward kernels serve the whole set.
+    import torch
+    rng = np.random.default_rng(77)
+    C, L, N = 2, 64, 6
+    ks = []
+    for i in range(80):
+        ln = int(rng.choice([9, 11]))
+        d = int(rng.integers(2, 7)) if ln == 9 else int(rng.integers(2, 7))
+        p = int(rng.integers(8 * d + 1, (ln - 1) * d + 1)) if (ln - 1) * d > 8 * d else 8 * d
+        m = int(rng.integers(1, 3))
+        ks.append(dict(dilation=d, padding=p, channels=sorted(rng.choice(C, m, replace=False).tolist()),
+                       weights=rng.normal(size=(m, ln)), bias=float(rng.uniform(0.5, 1.0))))
+    kp = kernels_from_lists(C, L, ks)
+    X = -np.abs(ar1_spike_series(78, N, C, L))          # negative samples: the bias alone wins in the padding
+    lam, shift = 10.0, 3.0
+    g = normal_array(79, (N, 2 * kp.K))
+    ref = oracle.forward(kp, X, lam=lam, shift=shift)
+    far_left = (ref.argmax - kp.padding[None, :]) < -8 * kp.dilation[None, :]
+    assert far_left.sum() >= 10                           # the case is exercised
+    p = rk.RocketParams.from_kernel_params(kp)
+    Xd = torch.from_numpy(X).cuda()
+    feat, arg = rk.rocket_transform_soft(p, Xd, lam, shift)
+    P.check_argmax(arg.cpu().numpy(), ref)
+    dW, db = rk.rocket_transform_soft_backward(p, Xd, lam, shift, torch.from_numpy(g).cuda(),
+                                               torch.from_numpy(ref.argmax.astype(np.int32)).cuda())
+    rdW, rdb = oracle.backward(kp, X, g, ref.argmax, lam=lam, shift=shift)
+    P.check_grads(dW.cpu().numpy(), db.cpu().numpy(), rdW, rdb)
+    P.check_grads(np.zeros(0), db.cpu().numpy(), np.zeros(0), rdb)
+    p.close()
