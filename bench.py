@@ -33,9 +33,37 @@ TRAIN = dict(N=32, C=20, L=50000, K=10000)           # soft forward + backward s
 PARAM_SEED, DATA_SEED, GRAD_SEED = 8527, 2301, 527
 LAMBDA, SHIFT = 10.0, 3.0
 
-# DRAM bytes (read + write) of one launch of the dominant kernel, from the committed ncu capture
-# (profiles/); None until a capture of the current kernel exists.
-NCU_DRAM_BYTES_PER_LAUNCH = {"fast_s_forward": 56.0e6, "fast_t_forward": 311.8e6}   # per launch = one chunk of 12 examples
+# DRAM bytes (read + write) of one launch of either fused kernel, from the committed ncu capture (profiles/),
+# per launch = one chunk of 12 examples.  The figures belong to one state of the kernel sources: they are
+# reported only while the digest of those sources still equals NCU_SOURCES_DIGEST, and as null otherwise.
+NCU_DRAM_BYTES_PER_LAUNCH = {"fast_s_forward": 56.0e6, "fast_t_forward": 311.8e6}
+NCU_SOURCES_DIGEST = "unset"
+KERNEL_SOURCES = ("rocket_fast_fwd.cu", "rocket_fast.h", "rocket_fast_geom.h", "rocket_plan.cpp")
+
+
+def kernel_sources_digest():
+    """Digest of the sources that decide what the fused kernels read and write."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2301_08527_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def measured_fma_peak():
+    """FP32 FMA rate of dependent register chains on this device (scalar and packed two-wide), measured with the
+    benchmark-only helper library; None when it cannot run."""
+    import ctypes
+    try:
+        from paper_2301_08527_b200.build import build_bench_helper
+        lib = ctypes.CDLL(build_bench_helper())
+        a, b = ctypes.c_double(0.0), ctypes.c_double(0.0)
+        if lib.fma_peak_measure(ctypes.byref(a), ctypes.byref(b)) != 0:
+            return None
+        return {"scalar_fma_tflops": a.value, "packed_fma_tflops": b.value}
+    except Exception:
+        return None
 
 
 def fp32_peak_tflops(sm_count, sm_mhz):
@@ -183,7 +211,9 @@ def main():
     ap.add_argument("--ref-kernels", type=int, default=2000, help="kernels per step of the reference arm's sample")
     ap.add_argument("--skip-passes", action="store_true", help="skip the soft forward / backward timings")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
-    ap.add_argument("--sweep", action="store_true", help="also time the throughput sweep (config 4) on rank 0")
+    ap.add_argument("--sweep", action="store_true", help="time the whole throughput sweep (config 4: 24 points, three timed "
+                    "calls each) on rank 0 instead of its time-boxed default (12 points, one timed call each)")
+    ap.add_argument("--skip-sweep", action="store_true", help="skip the throughput sweep")
     ap.add_argument("--small", action="store_true", help="profiling case: N=12 examples, one launch of either fused kernel")
     ap.add_argument("--profile-pass", choices=["soft", "backward"], default=None,
                     help="profiling case: run only that pass of config 3 on 12 examples, three times, and exit")
@@ -267,6 +297,7 @@ def main():
         per = [evs[i].elapsed_time(evs[i + 1]) * 1e-3 for i in range(steps)]
         return evs[0].elapsed_time(evs[-1]) * 1e-3, per
 
+    fma_peak = measured_fma_peak() if rank == 0 else None
     sampler = ClockSampler(local_rank) if rank == 0 else None
     launches0 = rk.kernel_launch_count()
     if sampler:
@@ -316,12 +347,14 @@ def main():
     peaks = measured_peaks()
     sm_max = (peaks or {}).get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
     peak = fp32_peak_tflops(props.multi_processor_count, sm_max)
+    traffic_valid = kernel_sources_digest() == NCU_SOURCES_DIGEST
     roofline = {"bound": "alu", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(dom.split()[0]),
+                "frac": achieved / peak,
+                "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(dom.split()[0]) if traffic_valid else None,
                 "launch_ms": dom_ms, "launches_per_step": chunk_launches,
-                "traffic_note": "ncu, cold cache, one launch = one chunk of 12 examples (48 MB of input)",
-                "peak_source": "derived: %d SMs x 128 FP32 lanes x 2 flop x %.0f MHz (max SM clock from %s); "
-                               "a packed-FMA microbenchmark reaches 74.0 TFLOP/s on this pool" % (
+                "traffic_note": ("ncu, cold cache, one launch = one chunk of 12 examples (48 MB of input)" if traffic_valid else
+                                 "null: the kernel sources changed since the committed ncu capture"),
+                "peak_source": "derived: %d SMs x 128 FP32 lanes x 2 flop x %.0f MHz (max SM clock from %s)" % (
                                    props.multi_processor_count, sm_max,
                                    "MEASURED_PEAKS.json" if peaks else "nvidia-smi / nominal"),
                 "flop_count": "2*len*channels*L_out per kernel per example; whole path %.4g flop/example, "
@@ -330,8 +363,15 @@ def main():
                             "fast_t_forward": {"ms": ms_t, "tflops": fl_t * w["N"] / (ms_t * 1e-3) / 1e12 if ms_t else None}},
                 "whole_step_tflops": step_tflops, "whole_step_frac": step_tflops / peak,
                 "pooling_ops_per_example": 2.0 * outputs_ex}
+    # the three denominators: lanes x maximum clock (peak / frac above), lanes x the clock observed during the timed
+    # steps, and the FMA rate a register-only chain microbenchmark reaches on this device in this run
     if clocks and clocks.get("sm_mhz"):
         roofline["frac_at_observed_clock"] = achieved / fp32_peak_tflops(props.multi_processor_count, clocks["sm_mhz"])
+    if fma_peak:
+        roofline["fma_microbenchmark"] = fma_peak
+        if fma_peak["packed_fma_tflops"] > 0:
+            roofline["frac_of_packed_fma_microbenchmark"] = achieved / fma_peak["packed_fma_tflops"]
+            roofline["whole_step_frac_of_packed_fma_microbenchmark"] = step_tflops / fma_peak["packed_fma_tflops"]
 
     passes = None
     if not args.skip_passes and not args.small:
@@ -343,6 +383,10 @@ def main():
         dW = torch.empty((params.n_weights,), dtype=torch.float32, device="cuda")
         db = torch.empty((t["K"],), dtype=torch.float32, device="cuda")
         psteps = max(2, args.steps // 3)
+        soft_by_lambda = {}
+        for lam in (1.0, 10.0, 100.0):     # config 3 sweeps the temperature; LAMBDA is the one quoted below
+            sl, _ = time_steps(lambda: rk.rocket_transform_soft(params, Xt, lam, SHIFT, out=sfeat, argmax_out=arg), psteps, 3)
+            soft_by_lambda[lam] = max_over(sl) / psteps
         s_soft, _ = time_steps(lambda: rk.rocket_transform_soft(params, Xt, LAMBDA, SHIFT, out=sfeat, argmax_out=arg),
                                psteps, 3)
         s_bwd, _ = time_steps(lambda: rk.rocket_transform_soft_backward(params, Xt, LAMBDA, SHIFT, g, arg, dW, db),
@@ -387,31 +431,37 @@ def main():
                         "e2e_examples_per_s": world * w["N"] / s_u8_e2e, "h2d_bytes_per_step": X8_host.numel()},
             "shape": "N=32 x C=20 x L=50000, K=10000 (config 3), lambda=%g, shift=%g" % (LAMBDA, SHIFT),
             "soft_forward": {"examples_per_s": world * t["N"] / s_soft, "ms": 1e3 * s_soft,
-                             "conv_tflops": flops_ex * t["N"] / s_soft / 1e12},
+                             "conv_tflops": flops_ex * t["N"] / s_soft / 1e12,
+                             "by_lambda": {"%g" % lam: {"ms": 1e3 * v, "examples_per_s": world * t["N"] / v,
+                                                        "conv_tflops": flops_ex * t["N"] / v / 1e12}
+                                           for lam, v in soft_by_lambda.items()}},
             "soft_backward": {"examples_per_s": world * t["N"] / s_bwd, "ms": 1e3 * s_bwd,
                               "conv_tflops": 2 * flops_ex * t["N"] / s_bwd / 1e12,
                               "flop_count": "4*len*channels*L_out (recompute z + dW)"},
         }
 
     sweep = None
-    if args.sweep and rank == 0:
+    if rank == 0 and not args.skip_sweep and not args.small:
         # config 4: hard transform, N in {1, 8, 60, 256} x L in {10k, 50k, 200k} x K in {10k, 50k}; N = 1 is the
-        # streaming latency.  Fresh inputs per (N, L); three timed calls after two warm-ups.
+        # streaming latency.  Inputs: eight generated examples per L, repeated up to N.  By default a time-boxed
+        # subset (N in {1, 60}, one timed call after one warm-up); --sweep times every point three times.
         sweep = []
+        batch_sizes, timed, warm = ((1, 8, 60, 256), 3, 2) if args.sweep else ((1, 60), 1, 1)
         for L4 in (10000, 50000, 200000):
+            X8 = torch.from_numpy(ar1_spike_series(DATA_SEED, 8, 20, L4)).cuda()
             for K4 in (10000, 50000):
                 p4 = rk.RocketParams.generate(PARAM_SEED, K4, 20, L4)
                 fl4, _ = p4.work()
-                for N4 in (1, 8, 60, 256):
-                    X4 = torch.from_numpy(ar1_spike_series(DATA_SEED, min(N4, 8), 20, L4)).cuda()
-                    X4 = X4.repeat((N4 + X4.shape[0] - 1) // X4.shape[0], 1, 1)[:N4].contiguous()
+                for N4 in batch_sizes:
+                    X4 = X8.repeat((N4 + 7) // 8, 1, 1)[:N4].contiguous()
                     f4 = torch.empty((N4, 2 * K4), dtype=torch.float32, device="cuda")
-                    t4, _ = time_steps(lambda: rk.rocket_transform(p4, X4, out=f4), 3, 2)
-                    t4 /= 3
+                    t4, _ = time_steps(lambda: rk.rocket_transform(p4, X4, out=f4), timed, warm)
+                    t4 /= timed
                     sweep.append({"N": N4, "L": L4, "K": K4, "ms": 1e3 * t4, "examples_per_s": N4 / t4,
-                                  "conv_tflops": fl4 * N4 / t4 / 1e12})
+                                  "conv_tflops": fl4 * N4 / t4 / 1e12, "timed_calls": timed})
                     del X4, f4
                 p4.close()
+            del X8
 
     cpu = None
     if rank == 0 and world == 1 and not args.skip_cpu_baseline:

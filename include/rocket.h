@@ -85,7 +85,8 @@ int rocket_params_generate(uint64_t seed, int K, int C, int L, rocket_params_t**
  * Requirements, else ROCKET_EINVAL: 1 <= length[k] <= 11; dilation[k] >= 1; padding[k] >= 0;
  * L_out,k >= 1; 1 <= num_channels[k] <= min(C, 11); channel indices of one kernel distinct and
  * in [0, C).  Any such kernel is accepted, up to L_out,k <= 2^30 (ROCKET_EUNSUPPORTED beyond);
- * lengths 7, 9 and 11 take the fast path.
+ * kernels of length 7, 9 or 11 are served by the fused kernels (for C <= 20 channels and L >= 16),
+ * every other kernel of the same handle by the generic ones, in every pass.
  */
 int rocket_params_from_arrays(int K, int C, int L, const int32_t* length, const int32_t* dilation,
                               const int32_t* padding, const int32_t* num_channels,
@@ -142,7 +143,9 @@ void rocket_params_destroy(rocket_params_t* p);
 
 /*
  * Hard transform: PPV (Eq. 1-2, strict z > 0) and max for every (example, kernel).
- *   X_dev    [N][C][L] fp32, device, 16-byte aligned;  C and L must equal the handle's
+ *   X_dev    [N][C][L] fp32, device (a 16-byte aligned base with L a multiple of 4 lets the staging copy
+ *            move 16 bytes at a time; any other base or length works, one float at a time);  C and L must
+ *            equal the handle's
  *   feat_dev [N][2K] fp32, device, written
  * N = 0 is a successful no-op.
  */
@@ -198,7 +201,7 @@ int rocket_transform_soft_backward_host(rocket_params_t* p, const float* X_host,
  * device; mean and inv_std are HOST arrays of C floats (statistics of the training set, not of the
  * batch) and are read before the call returns; outputs, stream, ownership and errors as in the fp32
  * forms, plus ROCKET_EINVAL for a NULL or NaN statistic.  When every kernel of the handle is served
- * by the fused kernels (lengths 7/9/11, L % 4 == 0, C <= 20) and X_u8_dev is 4-byte aligned, the
+ * by the fused kernels (lengths 7/9/11, C <= 20), L is a multiple of 4 and X_u8_dev is 4-byte aligned, the
  * scaling happens while the kernels' staging copy of the batch is written and no fp32 copy of the
  * batch exists; otherwise the call first writes a scaled fp32 copy into a buffer of the handle
  * (grown with cudaMalloc on demand, ROCKET_ENOMEM if that fails) and takes the fp32 route.

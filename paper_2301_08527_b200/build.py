@@ -56,5 +56,23 @@ def build(force=False, verbose=False):
     return LIB
 
 
+BENCH_SRC = os.path.join(HERE, "bench_csrc", "fma_peak.cu")
+BENCH_LIB = os.path.join(HERE, "libfma_peak_bench.so")
+
+
+def build_bench_helper(force=False):
+    """Compile the benchmark-only FMA-rate helper (bench_csrc/fma_peak.cu); returns its path.  It is no part
+    of librocket_b200.so: only bench.py loads it, to measure the FP32 FMA rate its roofline figures quote."""
+    if not force and os.path.exists(BENCH_LIB) and os.path.getmtime(BENCH_LIB) >= os.path.getmtime(BENCH_SRC):
+        return BENCH_LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    tmp = BENCH_LIB + ".%d.tmp" % os.getpid()
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
+                           "-Xcompiler", "-fPIC", BENCH_SRC, "-o", tmp, "-lcudart_static", "-lpthread", "-ldl", "-lrt"])
+    os.replace(tmp, BENCH_LIB)
+    return BENCH_LIB
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_bench_helper(force="--force" in sys.argv))

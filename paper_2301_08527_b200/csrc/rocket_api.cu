@@ -384,7 +384,7 @@ int rocket_transform(const rocket_params_t* p, const float* X_dev, int N, int C,
     DeviceGuard g(p->device);
     if (!g.ok) return ROCKET_ECUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const bool aligned = (reinterpret_cast<uintptr_t>(X_dev) & 15u) == 0;
+    const bool aligned = (reinterpret_cast<uintptr_t>(X_dev) & 3u) == 0;
     if (p->path == 0 && p->fast->host.enabled && aligned) {
         cudaError_t e = fast::launch_fast_forward(*p->fast, p->dp, X_dev, N, feat_dev, stream);
         if (e != cudaSuccess) return cuda_status(e);
@@ -406,7 +406,7 @@ int rocket_transform_soft(const rocket_params_t* p, const float* X_dev, int N, i
     DeviceGuard g(p->device);
     if (!g.ok) return ROCKET_ECUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const bool aligned = (reinterpret_cast<uintptr_t>(X_dev) & 15u) == 0;
+    const bool aligned = (reinterpret_cast<uintptr_t>(X_dev) & 3u) == 0;
     if (p->path == 0 && p->fast->host.enabled && aligned) {
         cudaError_t e = fast::launch_fast_forward(*p->fast, p->dp, X_dev, N, feat_dev, stream, true, lambda, shift, argmax_dev);
         if (e != cudaSuccess) return cuda_status(e);
@@ -433,7 +433,7 @@ static int transform_u8(const rocket_params_t* p, const uint8_t* X_u8_dev, int N
     DeviceGuard g(p->device);
     if (!g.ok) return ROCKET_ECUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const bool aligned = (reinterpret_cast<uintptr_t>(X_u8_dev) & 3u) == 0;
+    const bool aligned = (reinterpret_cast<uintptr_t>(X_u8_dev) & 3u) == 0 && L % 4 == 0;
     if (p->path == 0 && p->fast->host.enabled && p->fast->dev.n_generic == 0 && aligned && C <= fast::kNormMaxChannels) {
         // every kernel is served by the fused kernels: the scaling happens while their staging copy is written
         fast::NormArgs norm;
@@ -489,10 +489,15 @@ int rocket_transform_soft_backward(const rocket_params_t* p, const float* X_dev,
     if (!g.ok) return ROCKET_ECUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int64_t nW = n_weights_of(p);
-    const bool aligned = (reinterpret_cast<uintptr_t>(X_dev) & 15u) == 0;
-    if (p->path == 0 && p->fast->host.enabled && p->fast->host.generic_list.empty() && (aligned || N == 0))
-        return cuda_status(fast::launch_fast_backward(*p->fast, p->dp, nW, X_dev, N, lambda, shift, dfeat_dev, argmax_dev,
-                                                      dW_dev, db_dev, stream));
+    const bool aligned = (reinterpret_cast<uintptr_t>(X_dev) & 3u) == 0;
+    const bool use_fast = p->path == 0 && p->fast->host.enabled && (aligned || N == 0);
+    const int n_generic = use_fast ? (int)p->fast->host.generic_list.size() : p->host.K;
+    if (use_fast) {   // the fused kernels assign dW / db of the kernels they serve
+        cudaError_t e = fast::launch_fast_backward(*p->fast, p->dp, nW, X_dev, N, lambda, shift, dfeat_dev, argmax_dev,
+                                                   dW_dev, db_dev, stream);
+        if (e != cudaSuccess) return cuda_status(e);
+        if (n_generic == 0) return ROCKET_OK;
+    }
     float* scratch = nullptr;
     if (N > 0) {
         std::lock_guard<std::mutex> lk(p->mu);
@@ -501,7 +506,8 @@ int rocket_transform_soft_backward(const rocket_params_t* p, const float* X_dev,
         scratch = static_cast<float*>(p->scratch.ptr);
     }
     return cuda_status(launch_generic_backward(p->dp, nW, X_dev, N, lambda, shift, dfeat_dev, argmax_dev, scratch,
-                                               dW_dev, db_dev, stream));
+                                               dW_dev, db_dev, stream, use_fast ? p->fast->dev.generic_list : nullptr,
+                                               use_fast ? n_generic : 0));
 }
 
 // ---- host-buffer forms ----------------------------------------------------------------------

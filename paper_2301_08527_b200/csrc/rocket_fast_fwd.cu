@@ -118,6 +118,27 @@ __device__ __forceinline__ void pool_hard(const u64 (&acc)[kR], int& cnt, float&
     cnt += __popc(signs);
 }
 
+// The same for a warp tile with outputs that do not exist: m0 / m1 hold one bit per row of the thread's two
+// columns (bit o set: row o is an output); the others are replaced by +inf on the way (sign bit clear, neutral
+// for the min), so the accumulators may hold anything there.
+__device__ __forceinline__ void pool_hard_masked(const u64 (&acc)[kR], unsigned m0, unsigned m1, int& cnt, float& mn) {
+    const float inf = __int_as_float(0x7f800000);
+    unsigned signs = 0;
+#pragma unroll
+    for (int o = 0; o < kR; ++o) {
+        float a, b;
+        unpack2(acc[o], a, b);
+        a = (m0 & (1u << o)) ? a : inf;
+        b = (m1 & (1u << o)) ? b : inf;
+        signs = __funnelshift_l(__float_as_uint(a), signs, 1);
+        signs = __funnelshift_l(__float_as_uint(b), signs, 1);
+        mn = min3(mn, a, b);
+    }
+    cnt += __popc(signs);
+}
+// Bit o set for lo <= o < hi (0 <= lo, hi <= 16).
+__device__ __forceinline__ unsigned row_mask(int lo, int hi) { return hi > lo ? ((1u << hi) - 1u) & ~((1u << lo) - 1u) : 0u; }
+
 // Accumulators of a tile: 0 - bias where the output exists, +inf elsewhere.
 __device__ __forceinline__ void init_acc(u64 (&acc)[kR], float negb, bool interior, int lo0, int hi0, int lo1, int hi1) {
     if (interior) {
@@ -465,10 +486,13 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
                 interior = __all_sync(kFull, lo0 == 0 && lo1 == 0 && hi0 == kR && hi1 == kR);
             }
             u64 acc[kR];
-            if (!interior) init_acc(acc, rec->negb, false, lo0, hi0, lo1, hi1);
-            if (len == 7) s_kernel_tile<7>(planes, rec, lane, acc, interior);
-            else if (len == 9) s_kernel_tile<9>(planes, rec, lane, acc, interior);
-            else s_kernel_tile<11>(planes, rec, lane, acc, interior);
+            // hard mode: the pooling masks the outputs that do not exist, so the accumulators always start inside
+            // the first channel's pass; the other modes start them at +inf where there is no output
+            const bool fold = interior || MODE == 0;
+            if (!fold) init_acc(acc, rec->negb, false, lo0, hi0, lo1, hi1);
+            if (len == 7) s_kernel_tile<7>(planes, rec, lane, acc, fold);
+            else if (len == 9) s_kernel_tile<9>(planes, rec, lane, acc, fold);
+            else s_kernel_tile<11>(planes, rec, lane, acc, fold);
             if (MODE == 2) {
                 const int64_t pair = (int64_t)n * a.K + korig;
                 const float gP = __ldg(a.dfeat + 2 * pair), gM = __ldg(a.dfeat + 2 * pair + 1);
@@ -492,7 +516,8 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
             } else {
                 int cnt = 0;
                 float mn = __int_as_float(0x7f800000);
-                pool_hard(acc, cnt, mn);
+                if (interior) pool_hard(acc, cnt, mn);
+                else pool_hard_masked(acc, row_mask(lo0, hi0), row_mask(lo1, hi1), cnt, mn);
                 publish(a.feat_i, (int64_t)n * a.K + korig, cnt, mn, lane);
             }
             __syncwarp();  // every lane is done with the record before its slot is refilled
@@ -807,9 +832,11 @@ __global__ void __launch_bounds__(kTBlockThreads, kTBlocksPerSM) fast_t_forward(
                               : t_box_offset(cg, k, box_rows) + 4 * wr * boxw + lc;
             const int gl = si.g_lo, gh = si.g_hi;
             u64 acc[kR];
-            // interior warp tiles of ordinary tiles start their accumulators inside the first channel's pass
-            const bool fold = interior && !wide;
-            if (active && !fold) init_acc(acc, rec->negb, interior, lo0, hi0, lo1, hi1);
+            // Ordinary tiles start their accumulators inside the first channel's pass: interior warp tiles in every
+            // mode, the others in hard mode, where the pooling masks the outputs that do not exist.  Everywhere
+            // else the accumulators start at 0 - bias, or +inf where there is no output.
+            const bool fold = !wide && (interior || MODE == 0);
+            if (active && !fold) init_acc(acc, rec->negb, interior || MODE == 0, lo0, hi0, lo1, hi1);
             if (wide) ok = t_dispatch<kTWideCols, true>(len, stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh, false);
             else if (cg == 1) ok = t_dispatch<kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0, fold);
             else if (cg == 2) ok = t_dispatch<2 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0, fold);
@@ -850,7 +877,8 @@ __global__ void __launch_bounds__(kTBlockThreads, kTBlocksPerSM) fast_t_forward(
                         cnt = 0;
                         mn = __int_as_float(0x7f800000);
                     }
-                    pool_hard(acc, cnt, mn);
+                    if (interior) pool_hard(acc, cnt, mn);
+                    else pool_hard_masked(acc, row_mask(lo0, hi0), row_mask(lo1, hi1), cnt, mn);
                 }
             }
             ++it;
@@ -885,6 +913,21 @@ __global__ void fast_pad_copy_kernel(const float4* __restrict__ X, float* __rest
             float* dj = dst + j * copy_floats - j;
             dj[0] = v.x; dj[1] = v.y; dj[2] = v.z; dj[3] = v.w;
         }
+    }
+}
+
+// The same for series whose length is not a multiple of four floats, or whose base is not 16-byte aligned:
+// one float per thread and step.
+__global__ void fast_pad_copy_scalar_kernel(const float* __restrict__ X, float* __restrict__ xpad, int64_t rows, int L,
+                                            int64_t pitch, int front, int64_t copy_floats) {
+    const int64_t total = rows * L;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t rho = e / L;
+        const int i = (int)(e - rho * L);
+        const float v = __ldg(X + e);
+        float* dst = xpad + rho * pitch + front + i;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dst[j * copy_floats - j] = v;
     }
 }
 
@@ -999,6 +1042,15 @@ cudaError_t set_kernel_attributes(int dev) {
 
 // ---- backward helpers ----------------------------------------------------------------------------
 // Largest |x| of the batch, as the bit pattern of a non-negative float (integer order = float order).
+__global__ void fast_absmax_scalar_kernel(const float* __restrict__ X, int64_t n, unsigned* __restrict__ out) {
+    float m = 0.0f;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x)
+        m = fmaxf(m, fabsf(__ldg(X + e)));
+    unsigned b = __float_as_uint(m);
+    b = __reduce_max_sync(kFull, b);
+    if ((threadIdx.x & 31) == 0) atomicMax(out, b);
+}
+
 __global__ void fast_absmax_kernel(const float4* __restrict__ X, int64_t n4, unsigned* __restrict__ out) {
     float m = 0.0f;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n4; e += (int64_t)gridDim.x * blockDim.x) {
@@ -1149,6 +1201,16 @@ cudaError_t ensure_pad_capacity(FastState& fs, int N, int C, int L, bool without
     return cudaSuccess;
 }
 
+// Writes `rows` channel rows of X into the four shifted zero-margined copies (16-byte pieces when the rows allow).
+static void launch_pad_copy(FastState& fs, const float* X, int64_t rows, int L, int sms, cudaStream_t stream) {
+    if (L % 4 == 0 && (reinterpret_cast<uintptr_t>(X) & 15u) == 0)
+        fast_pad_copy_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(X), fs.xpad, rows, L / 4, fs.host.pad_pitch,
+                                                          kTPadFront, fs.copy_floats);
+    else
+        fast_pad_copy_scalar_kernel<<<sms * 8, 256, 0, stream>>>(X, fs.xpad, rows, L, fs.host.pad_pitch, kTPadFront, fs.copy_floats);
+    count_launch();
+}
+
 // Soft transform: 16 bytes per (example, kernel), grow-only.
 static cudaError_t ensure_soft_ws(FastState& fs, int64_t pairs) {
     if ((size_t)pairs * 16 <= fs.soft_ws_bytes) return cudaSuccess;
@@ -1182,7 +1244,7 @@ cudaError_t reserve_fast_state(FastState& fs, const DeviceParams& dp, int max_N,
         if (e != cudaSuccess) return e;
     }
     if (soft && (e = ensure_soft_ws(fs, (int64_t)max_N * dp.K)) != cudaSuccess) return e;
-    if (backward && fs.host.generic_list.empty() && (e = ensure_bwd_ws(fs, dp, n_weights)) != cudaSuccess) return e;
+    if (backward && (e = ensure_bwd_ws(fs, dp, n_weights)) != cudaSuccess) return e;
     return cudaSuccess;
 }
 
@@ -1248,9 +1310,7 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
                 fs.host.pad_pitch, kTPadFront, fs.copy_floats, *norm);
             count_launch();
         } else if (pd.n_titems > 0) {
-            fast_pad_copy_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(a.X), fs.xpad, (int64_t)nc * dp.C,
-                                                              dp.L / 4, fs.host.pad_pitch, kTPadFront, fs.copy_floats);
-            count_launch();
+            launch_pad_copy(fs, a.X, (int64_t)nc * dp.C, dp.L, sms, stream);
         }
         if (fs.profile) cudaEventRecord(fs.evs[3 * c], stream);
         if (pd.n_sitems > 0) {
@@ -1306,9 +1366,11 @@ cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t 
     }
     e = cudaMemsetAsync(absmax, 0, 256, stream);
     if (e != cudaSuccess) return e;
-    const int64_t n4 = (int64_t)N * dp.C * (dp.L / 4);
-    if (n4 > 0) {
-        fast_absmax_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(X), n4, absmax);
+    const int64_t n_x = (int64_t)N * dp.C * dp.L;
+    if (n_x > 0) {
+        if (dp.L % 4 == 0 && (reinterpret_cast<uintptr_t>(X) & 15u) == 0)
+            fast_absmax_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(X), n_x / 4, absmax);
+        else fast_absmax_scalar_kernel<<<sms * 8, 256, 0, stream>>>(X, n_x, absmax);
         count_launch();
     }
     fast_bwd_prepare_kernel<<<(pd.n_krec + 127) / 128, 128, 0, stream>>>(dfeat, pd.krec, pd.n_krec, N, dp.K, lambda, absmax, scale,
@@ -1328,11 +1390,7 @@ cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t 
         a.N = nc;
         e = cudaMemsetAsync(pd.counters, 0, 8, stream);
         if (e != cudaSuccess) return e;
-        if (pd.n_titems > 0) {
-            fast_pad_copy_kernel<<<sms * 8, 256, 0, stream>>>(reinterpret_cast<const float4*>(a.X), fs.xpad, (int64_t)nc * dp.C,
-                                                              dp.L / 4, fs.host.pad_pitch, kTPadFront, fs.copy_floats);
-            count_launch();
-        }
+        if (pd.n_titems > 0) launch_pad_copy(fs, a.X, (int64_t)nc * dp.C, dp.L, sms, stream);
         if (pd.n_sitems > 0) {
             const unsigned long long total = (unsigned long long)nc * pd.n_sitems;
             const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms);

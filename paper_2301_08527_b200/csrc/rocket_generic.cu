@@ -102,14 +102,15 @@ constexpr int kTile = 1024;  // outputs whose gz is held in shared memory at a t
 __global__ void __launch_bounds__(kThreads)
 generic_backward_kernel(DeviceParams dp, int64_t n_weights, const float* __restrict__ X, float lambda,
                         float shift, const float* __restrict__ dfeat, const int32_t* __restrict__ argmax,
-                        float* __restrict__ scratch) {
+                        float* __restrict__ scratch, const int32_t* __restrict__ klist, int nk) {
     __shared__ float sW[kMaxTaps];
     __shared__ int sS[ROCKET_MAX_CHANNELS_PER_KERNEL];
     __shared__ float sgz[kTile];
     __shared__ float rdb[kWarps];
 
     const int64_t e = blockIdx.x;
-    const int n = (int)(e / dp.K), k = (int)(e % dp.K);
+    const int n = (int)(e / nk);
+    const int k = klist ? klist[e % nk] : (int)(e % nk);
     const KernelShape s = load_kernel(dp, k, sW, sS);
     const float* Xn = X + (int64_t)n * dp.C * dp.L;
     const float b = dp.bias[k];
@@ -186,6 +187,23 @@ reduce_examples_kernel(const float* __restrict__ scratch, int N, int64_t n_weigh
     else db[t - n_weights] = a;
 }
 
+// The same sum for a list of kernels only (one block per listed kernel): the other entries of dW / db belong
+// to someone else and are left alone.
+__global__ void __launch_bounds__(kThreads)
+reduce_examples_list_kernel(const float* __restrict__ scratch, int N, int64_t n_weights, DeviceParams dp,
+                            const int32_t* __restrict__ klist, float* __restrict__ dW, float* __restrict__ db) {
+    const int k = klist[blockIdx.x];
+    const int64_t width = n_weights + dp.K;
+    const int wo = dp.weight_offset[k], taps = dp.weight_offset[k + 1] - wo;
+    for (int t = threadIdx.x; t <= taps; t += kThreads) {
+        const int64_t col = t < taps ? (int64_t)wo + t : n_weights + k;
+        float a = 0.0f;
+        for (int n = 0; n < N; ++n) a += scratch[(int64_t)n * width + col];
+        if (t < taps) dW[wo + t] = a;
+        else db[k] = a;
+    }
+}
+
 // Per-channel feature scaling of raw 8-bit intensities (Sections 4.1 and 4.3).
 __global__ void __launch_bounds__(kThreads)
 normalise_u8_kernel(const uint8_t* __restrict__ X, int64_t total, int L, int C, const float* __restrict__ mean,
@@ -227,19 +245,26 @@ size_t generic_backward_scratch_floats(int N, int64_t n_weights, int K) {
 
 cudaError_t launch_generic_backward(const DeviceParams& dp, int64_t n_weights, const float* X, int N,
                                     float lambda, float shift, const float* dfeat, const int32_t* argmax,
-                                    float* scratch, float* dW, float* db, cudaStream_t stream) {
-    const int64_t blocks = (int64_t)N * dp.K;
+                                    float* scratch, float* dW, float* db, cudaStream_t stream, const int32_t* klist,
+                                    int nk) {
+    if (!klist) nk = dp.K;
+    if (nk == 0) return cudaSuccess;
+    const int64_t blocks = (int64_t)N * nk;
     if (blocks > 0x7fffffffll) return cudaErrorInvalidConfiguration;
     if (blocks > 0) {
         generic_backward_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(dp, n_weights, X, lambda, shift, dfeat,
-                                                                           argmax, scratch);
+                                                                           argmax, scratch, klist, nk);
         count_launch();
         cudaError_t err = cudaGetLastError();
         if (err != cudaSuccess) return err;
     }
-    const int64_t width = n_weights + dp.K;
-    reduce_examples_kernel<<<(unsigned)((width + kThreads - 1) / kThreads), kThreads, 0, stream>>>(
-        scratch, N, n_weights, dp.K, dW, db);
+    if (klist) {
+        reduce_examples_list_kernel<<<(unsigned)nk, kThreads, 0, stream>>>(scratch, N, n_weights, dp, klist, dW, db);
+    } else {
+        const int64_t width = n_weights + dp.K;
+        reduce_examples_kernel<<<(unsigned)((width + kThreads - 1) / kThreads), kThreads, 0, stream>>>(
+            scratch, N, n_weights, dp.K, dW, db);
+    }
     count_launch();
     return cudaGetLastError();
 }

@@ -60,9 +60,11 @@ size_t generic_backward_scratch_floats(int N, int64_t n_weights, int K);
 // x[i] = (v[i] - mean[c]) * inv_std[c] for [rows][L] 8-bit samples, c = row % C (mean, inv_std on the device).
 cudaError_t launch_normalise_u8(const uint8_t* X, int64_t rows, int L, int C, const float* mean, const float* inv_std,
                                 float* out, cudaStream_t stream);
+// klist (device, nk entries) restricts the pass to those kernels, whose dW / db entries alone are written.
 cudaError_t launch_generic_backward(const DeviceParams& dp, int64_t n_weights, const float* X, int N,
                                     float lambda, float shift, const float* dfeat, const int32_t* argmax,
-                                    float* scratch, float* dW, float* db, cudaStream_t stream);
+                                    float* scratch, float* dW, float* db, cudaStream_t stream,
+                                    const int32_t* klist = nullptr, int nk = 0);
 
 }  // namespace rocket
 

@@ -28,9 +28,10 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
     if (split < kTMinDilation) split = kTMinDilation;
     out.split = split;
     const int K = hp.K;
-    // The fast kernels want 16-byte aligned channel rows and at most kSMaxChannels channels in
-    // an S tile.
-    const bool shape_ok = (hp.L % 4 == 0) && hp.C <= kSMaxChannels && hp.L >= 16;
+    // The fast kernels stage at most kSMaxChannels channels in an S tile.  Any series length will do: the
+    // small-dilation kernel copies single floats and the large-dilation kernel reads the zero-margined
+    // copies, whose pitch does not depend on L.
+    const bool shape_ok = hp.C <= kSMaxChannels && hp.L >= 16;
     std::vector<int> s_kernels, t_kernels;
     for (int k = 0; k < K; ++k) {
         const int len = hp.length[k], d = hp.dilation[k];

@@ -207,6 +207,8 @@ int main() {
     rc |= check(13, 300, 3, 1000, 64);
     rc |= check(14, 200, 2, 16, 64);
     rc |= check(21, 300, 20, 200000, 64);
+    rc |= check(22, 300, 5, 4099, 64);      // series lengths that are no multiple of four floats
+    rc |= check(23, 200, 20, 50001, 64);
     // hand-made kernels: padding that is not a multiple of the dilation, extreme dilations, tiny outputs
     HostParams hp;
     hp.K = 0; hp.C = 2; hp.L = 1000;

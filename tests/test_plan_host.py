@@ -17,4 +17,4 @@ def test_plan_covers_every_output_once_and_copies_stay_in_bounds(tmp_path):
     subprocess.check_call(cmd)
     out = subprocess.run([exe], capture_output=True, text=True)
     assert out.returncode == 0, out.stdout + out.stderr
-    assert out.stdout.count("ok seed") == 8
+    assert out.stdout.count("ok seed") == 10
