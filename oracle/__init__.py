@@ -14,17 +14,18 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "rocket_oracle.c")
+_SRC_MINI = os.path.join(_HERE, "minirocket_oracle.c")
 _LIB = os.path.join(_HERE, "_build", "librocket_oracle.so")
 _lib = None
 
 
 def build(force=False):
     """Compile the oracle with gcc (-O2, OpenMP).  Returns the path of the shared object."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_MINI)):
         os.makedirs(os.path.dirname(_LIB), exist_ok=True)
         tmp = _LIB + ".%d.tmp" % os.getpid()
         subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
-                               "-ffp-contract=off", "-o", tmp, _SRC, "-lm"])
+                               "-ffp-contract=off", "-o", tmp, _SRC, _SRC_MINI, "-lm"])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -43,6 +44,7 @@ def _load():
     if _lib is None:
         lib = ctypes.CDLL(build())
         lib.rocket_oracle_conv.restype = ctypes.c_int64
+        lib.minirocket_oracle_conv.restype = ctypes.c_int64
         lib.rocket_oracle_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -195,3 +197,70 @@ def backward(p, X, g, argmax, lam=1.0, shift=3.0, examples=None, kernels=None):
                                _ptr(ks), ctypes.c_double(lam), ctypes.c_double(shift), _ptr(g), _ptr(argmax),
                                _ptr(dW), _ptr(db))
     return dW, db
+
+
+# ---- MINIROCKET (oracle/minirocket_oracle.c) ---------------------------------------------------------------
+
+class _CMini(ctypes.Structure):
+    _fields_ = [("C", ctypes.c_int), ("L", ctypes.c_int), ("F", ctypes.c_int), ("n_combos", ctypes.c_int),
+                ("taps", ctypes.c_void_p), ("dilation", ctypes.c_void_p), ("kernel_index", ctypes.c_void_p),
+                ("padded", ctypes.c_void_p), ("num_channels", ctypes.c_void_p), ("channel_idx", ctypes.c_void_p),
+                ("channel_offset", ctypes.c_void_p), ("feature_offset", ctypes.c_void_p)]
+
+
+def _cmini(p):
+    arrs = dict(taps=np.ascontiguousarray(p.taps, np.int32), dilation=np.ascontiguousarray(p.dilation, np.int32),
+                kernel_index=np.ascontiguousarray(p.kernel_index, np.int32), padded=np.ascontiguousarray(p.padded, np.int32),
+                num_channels=np.ascontiguousarray(p.num_channels, np.int32),
+                channel_idx=np.ascontiguousarray(p.channel_idx, np.int32),
+                channel_offset=np.ascontiguousarray(p.channel_offset, np.int64),
+                feature_offset=np.ascontiguousarray(p.feature_offset, np.int32))
+    s = _CMini(C=p.C, L=p.L, F=p.F, n_combos=p.n_combos, **{k: v.ctypes.data for k, v in arrs.items()})
+    return s, arrs
+
+
+def minirocket_conv(p, X, n, c):
+    """Convolution outputs of combination c on example n over the combination's output range, float64."""
+    lib = _load()
+    X = _check_x(p, X)
+    s, keep = _cmini(p)
+    nout = lib.minirocket_oracle_conv(ctypes.byref(s), _ptr(X), ctypes.c_int(n), ctypes.c_int(c), None)
+    z = np.empty(int(nout), dtype=np.float64)
+    lib.minirocket_oracle_conv(ctypes.byref(s), _ptr(X), ctypes.c_int(n), ctypes.c_int(c), _ptr(z))
+    return z
+
+
+def minirocket_example_index(p, N):
+    """Which of N training examples every combination reads its biases from."""
+    return np.minimum((p.example_draw * N).astype(np.int64), N - 1).astype(np.int32)
+
+
+def minirocket_fit(p, X):
+    """Biases [F] (float64) from the quantiles of the training examples' convolution outputs."""
+    lib = _load()
+    X = _check_x(p, X)
+    s, keep = _cmini(p)
+    ex = minirocket_example_index(p, X.shape[0])
+    q = np.ascontiguousarray(p.quantile, np.float64)
+    bias = np.empty(p.F, dtype=np.float64)
+    lib.minirocket_oracle_fit(ctypes.byref(s), _ptr(X), _ptr(ex), _ptr(q), _ptr(bias))
+    return bias
+
+
+def minirocket_transform(p, X, bias, eps=1e-5):
+    """PPV features [N, F] against the biases, and the counts that bound what fp32 arithmetic may decide
+    differently: pos_eps = #{z > bias + eps}, amb = #{|z - bias| <= eps}, n_out [F] = outputs per feature."""
+    lib = _load()
+    X = _check_x(p, X)
+    s, keep = _cmini(p)
+    N = X.shape[0]
+    bias = np.ascontiguousarray(bias, np.float64)
+    out = SimpleNamespace(ppv=np.empty((N, p.F)), pos_eps=np.empty((N, p.F), np.int64), amb=np.empty((N, p.F), np.int64))
+    lib.minirocket_oracle_transform(ctypes.byref(s), _ptr(X), ctypes.c_int(N), _ptr(bias), ctypes.c_double(eps),
+                                    _ptr(out.ppv), _ptr(out.pos_eps), _ptr(out.amb))
+    n_out = np.empty(p.F, np.int64)
+    for c in range(p.n_combos):
+        first, last = p.out_range(c)
+        n_out[p.feature_offset[c]:p.feature_offset[c + 1]] = last - first
+    out.n_out = n_out
+    return out

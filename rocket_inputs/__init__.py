@@ -7,11 +7,12 @@ parameters drawn by the rules of Section 3.1); none of the transform's arithmeti
 """
 from .rng import counter_u64, counter_uniform
 from .kernels import KernelParams, generate_kernels, kernels_from_lists
+from .minirocket import MiniParams, generate_minirocket
 from .series import (random_walk_series, ar1_spike_series, normal_array, intensity_series_u8,
                      channel_statistics)
 
 __all__ = [
     "counter_u64", "counter_uniform", "KernelParams", "generate_kernels",
     "kernels_from_lists", "random_walk_series", "ar1_spike_series", "normal_array",
-    "intensity_series_u8", "channel_statistics",
+    "intensity_series_u8", "channel_statistics", "MiniParams", "generate_minirocket",
 ]
