@@ -318,6 +318,50 @@ int rocket_transform_soft_backward_noalloc(const rocket_params_t* p, const float
                                            const int32_t* argmax_dev, float* dW_dev, float* db_dev,
                                            void* cuda_stream);
 
+/*
+ * MINIROCKET (Section 2: the model that followed ROCKET - two-valued kernels from a fixed set, so that the
+ * convolution needs additions only, biases sampled from the input data, PPV as the only pooled feature;
+ * Section 6 names it as the extension of the GPU implementation).
+ *
+ * What the paper leaves open is fixed as follows.  Kernels: the 84 ways to give three of nine taps the weight
+ * 2 and the other six -1.  num_features is rounded down to a multiple of 84 (10,000 -> 9,996); every kernel
+ * owns the same number of features, spread over the distinct values of floor(2^x), x equally spaced on
+ * [0, log2((L - 1) / 8)] (at most 32 of them).  Combination c = dilation_index * 84 + kernel_index owns the
+ * features feature_offset[c] .. feature_offset[c + 1] - 1, has padding 4 d (outputs 0 .. L - 1) when
+ * dilation_index + kernel_index is even and none otherwise (outputs 4 d .. L - 4 d - 1), and a random subset of
+ * floor(2^U(0, log2(min(C, 9) + 1))) channels whose samples are summed before the convolution (the same
+ * weights apply to every channel).  Feature f is
+ *     #{ i : z_i > bias_f } / number of outputs,   z_i = sum_{c in S} sum_{j<9} w_j xpad[c][i + (j - 4) d]
+ * and bias_f is the quantile frac((f + 1) / golden ratio) - linear interpolation between order statistics -
+ * of the outputs of training example floor(example_draw[c] * N).
+ *
+ * rocket_mini_create   host only; *out owns the parameters (release with rocket_mini_destroy).  Needs C >= 1,
+ *                      L >= 9, num_features >= 84.
+ * rocket_mini_fit      X_host [N][C][L] fp32 on the HOST; computes every bias (a one-off over one example per
+ *                      combination, on the host's cores); returns when done.
+ * rocket_mini_set_biases  installs biases computed elsewhere ([n_features] floats, host).
+ * rocket_mini_transform   X_dev [N][C][L] fp32 and feat_dev [N][n_features] fp32 on the device; one fused kernel
+ *                      on the caller's stream (convolution outputs never reach memory); the first call binds
+ *                      the handle to the current device and uploads its parameters.  ROCKET_EINVAL before
+ *                      a fit or set_biases; ROCKET_ESHAPE when C or L differ from the handle's.
+ * rocket_mini_host_view   read-only views of the host arrays (taps [84][3], per combination: dilation,
+ *                      kernel_index, padded, num_channels, ragged channel_idx, feature_offset [n + 1],
+ *                      example_draw; per feature: quantile, bias); any output pointer may be NULL.
+ */
+typedef struct rocket_mini rocket_mini_t;
+int rocket_mini_create(uint64_t seed, int C, int L, int num_features, rocket_mini_t** out);
+int rocket_mini_counts(const rocket_mini_t* p, int* C, int* L, int* n_features, int* n_combinations,
+                       int64_t* n_channel_idx);
+int rocket_mini_host_view(const rocket_mini_t* p, const int32_t** taps, const int32_t** dilation,
+                          const int32_t** kernel_index, const int32_t** padded, const int32_t** num_channels,
+                          const int32_t** channel_idx, const int32_t** feature_offset, const double** example_draw,
+                          const double** quantile, const float** bias);
+int rocket_mini_fit(rocket_mini_t* p, const float* X_host, int N);
+int rocket_mini_set_biases(rocket_mini_t* p, const float* bias);
+int rocket_mini_transform(const rocket_mini_t* p, const float* X_dev, int N, int C, int L, float* feat_dev,
+                          void* cuda_stream);
+void rocket_mini_destroy(rocket_mini_t* p);
+
 #ifdef __cplusplus
 }
 #endif

@@ -42,6 +42,15 @@ SIGNATURES = {
     "rocket_params_reserve": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_int]),
     "rocket_params_set_profiling": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
     "rocket_params_last_profile": (ctypes.c_int, [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_double)] * 4),
+    "rocket_mini_create": (ctypes.c_int, [ctypes.c_uint64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                          ctypes.POINTER(ctypes.c_void_p)]),
+    "rocket_mini_counts": (ctypes.c_int, [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_int)] * 4 + [ctypes.POINTER(ctypes.c_int64)]),
+    "rocket_mini_host_view": (ctypes.c_int, [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_void_p)] * 10),
+    "rocket_mini_fit": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]),
+    "rocket_mini_set_biases": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
+    "rocket_mini_transform": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                             ctypes.c_void_p, ctypes.c_void_p]),
+    "rocket_mini_destroy": (None, [ctypes.c_void_p]),
     "rocket_transform": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                         ctypes.c_void_p, ctypes.c_void_p]),
     "rocket_transform_soft": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
@@ -415,3 +424,77 @@ def rocket_transform_soft_backward_host(params, X_host, lam, shift, dfeat_host, 
         _host_ptr(argmax_host, torch.int32, "argmax_host"), _host_ptr(dW_host, torch.float32, "dW_host"),
         _host_ptr(db_host, torch.float32, "db_host")), "rocket_transform_soft_backward_host")
     return dW_host, db_host
+
+
+class MiniRocket:
+    """Owner of a rocket_mini_t handle (MINIROCKET parameters on host and device)."""
+
+    def __init__(self, handle):
+        self._h = handle
+        lib = load_library()
+        C, L, F, nc = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+        nch = ctypes.c_int64()
+        _check(lib.rocket_mini_counts(self._h, ctypes.byref(C), ctypes.byref(L), ctypes.byref(F), ctypes.byref(nc),
+                                      ctypes.byref(nch)), "rocket_mini_counts")
+        self.C, self.L, self.F, self.n_combos, self.n_channel_idx = C.value, L.value, F.value, nc.value, nch.value
+
+    @classmethod
+    def create(cls, seed, C, L, num_features=10000):
+        h = ctypes.c_void_p()
+        _check(load_library().rocket_mini_create(ctypes.c_uint64(seed), C, L, num_features, ctypes.byref(h)), "rocket_mini_create")
+        return cls(h)
+
+    def host_arrays(self):
+        """Copies of the handle's host arrays as a dict of numpy arrays."""
+        ptrs = [ctypes.c_void_p() for _ in range(10)]
+        _check(load_library().rocket_mini_host_view(self._h, *[ctypes.byref(q) for q in ptrs]), "rocket_mini_host_view")
+        names = ["taps", "dilation", "kernel_index", "padded", "num_channels", "channel_idx", "feature_offset",
+                 "example_draw", "quantile", "bias"]
+        sizes = [84 * 3, self.n_combos, self.n_combos, self.n_combos, self.n_combos, self.n_channel_idx, self.n_combos + 1,
+                 self.n_combos, self.F, self.F]
+        types = [np.int32] * 7 + [np.float64, np.float64, np.float32]
+        out = {}
+        for name, q, n, t in zip(names, ptrs, sizes, types):
+            ct = {np.int32: ctypes.c_int32, np.float64: ctypes.c_double, np.float32: ctypes.c_float}[t]
+            out[name] = np.ctypeslib.as_array(ctypes.cast(q, ctypes.POINTER(ct)), shape=(n,)).copy() if n else np.zeros(0, t)
+        out["taps"] = out["taps"].reshape(84, 3)
+        return out
+
+    def fit(self, X_host):
+        """Biases from the training examples X_host [N, C, L] (numpy float32, host)."""
+        X = np.ascontiguousarray(X_host, dtype=np.float32)
+        if X.ndim != 3 or X.shape[1] != self.C or X.shape[2] != self.L:
+            raise ValueError("X must be [N, %d, %d]" % (self.C, self.L))
+        _check(load_library().rocket_mini_fit(self._h, _np_ptr(X), X.shape[0]), "rocket_mini_fit")
+
+    def set_biases(self, bias):
+        b = np.ascontiguousarray(bias, dtype=np.float32)
+        if b.shape != (self.F,):
+            raise ValueError("one bias per feature")
+        _check(load_library().rocket_mini_set_biases(self._h, _np_ptr(b)), "rocket_mini_set_biases")
+
+    def transform(self, X, out=None):
+        """PPV features [N, F] of a CUDA float32 tensor X [N, C, L]."""
+        import torch
+        _check_x(self, X)
+        N = X.shape[0]
+        if out is None:
+            out = torch.empty((N, self.F), dtype=torch.float32, device=X.device)
+        _check(load_library().rocket_mini_transform(self._h, _dev_ptr(X, torch.float32, "X"), N, self.C, self.L,
+                                                    _dev_ptr(out, torch.float32, "out"), _stream()), "rocket_mini_transform")
+        return out
+
+    @property
+    def handle(self):
+        return self._h
+
+    def close(self):
+        if self._h:
+            load_library().rocket_mini_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
