@@ -90,13 +90,19 @@ mini_transform_kernel(const float* __restrict__ X, int C, int L, const MiniItem*
     const float* __restrict__ chan[kLen];
 #pragma unroll
     for (int q = 0; q < kLen; ++q) chan[q] = Xn + (size_t)it.ch[q < m ? q : 0] * L;
-    auto sample = [&](int row, int r) -> float {   // sum of the chosen channels at (row, r); zero outside the series
-        const long long pos = (long long)row * d + r;
-        if (row < 0 || pos >= L) return 0.0f;
-        float v = 0.0f;
-#pragma unroll
-        for (int q = 0; q < kLen; ++q)
-            if (q < m) v += __ldg(chan[q] + pos);
+    // sum of the chosen channels at sample pos; zero outside the series (the nesting keeps the number of
+    // executed loads at the number of channels: m is the same for the whole block)
+    auto sample_at = [&](int pos) -> float {
+        if ((unsigned)pos >= (unsigned)L) return 0.0f;
+        float v = __ldg(chan[0] + pos);
+        if (m > 1) { v += __ldg(chan[1] + pos);
+        if (m > 2) { v += __ldg(chan[2] + pos);
+        if (m > 3) { v += __ldg(chan[3] + pos);
+        if (m > 4) { v += __ldg(chan[4] + pos);
+        if (m > 5) { v += __ldg(chan[5] + pos);
+        if (m > 6) { v += __ldg(chan[6] + pos);
+        if (m > 7) { v += __ldg(chan[7] + pos);
+        if (m > 8) { v += __ldg(chan[8] + pos); } } } } } } } }
         return v;
     };
     const int nf = it.nf;
@@ -118,16 +124,7 @@ mini_transform_kernel(const float* __restrict__ X, int C, int L, const MiniItem*
         for (int p0 = first; p0 < last; p0 += kChunk) {
             const int lo = p0 - 4 * d, n_stage = min(kChunk, last - p0) + 8 * d;
             __syncthreads();
-            for (int e = threadIdx.x; e < n_stage; e += kThreads) {
-                const int pos = lo + e;
-                float v = 0.0f;
-                if (pos >= 0 && pos < L) {
-#pragma unroll
-                    for (int q = 0; q < kLen; ++q)
-                        if (q < m) v += __ldg(chan[q] + pos);
-                }
-                s_x[e] = v;
-            }
+            for (int e = threadIdx.x; e < n_stage; e += kThreads) s_x[e] = sample_at(lo + e);
             __syncthreads();
             const int n_out = min(kChunk, last - p0);
             for (int e = threadIdx.x; e < n_out; e += kThreads) {
@@ -142,20 +139,23 @@ mini_transform_kernel(const float* __restrict__ X, int C, int L, const MiniItem*
     for (int u = threadIdx.x; u < n_units; u += kThreads) {
         const int seg = u / d, r = u - seg * d;
         const int t_a = seg * rows_per_seg, t_b = min(T, t_a + rows_per_seg);
+        // every position of the walk fits 32 bits: (T + 8) d <= L + 9 d
         float win[kLen];
+        int pos = (t_a - 4) * d + r;                 // the sample the next window entry comes from
 #pragma unroll
-        for (int j = 0; j < kLen - 1; ++j) win[j + 1] = sample(t_a - 4 + j, r);
+        for (int j = 0; j < kLen - 1; ++j) { win[j + 1] = sample_at(pos); pos += d; }
+        int i = t_a * d + r;                         // the output the window is centred on next
         for (int t0 = t_a; t0 < t_b; t0 += kStep) {
             float nxt[kStep];
 #pragma unroll
-            for (int k = 0; k < kStep; ++k) nxt[k] = sample(t0 + 4 + k, r);
+            for (int k = 0; k < kStep; ++k) { nxt[k] = sample_at(pos); pos += d; }
 #pragma unroll
             for (int k = 0; k < kStep; ++k) {
 #pragma unroll
                 for (int j = 0; j < kLen - 1; ++j) win[j] = win[j + 1];
                 win[kLen - 1] = nxt[k];
-                const long long i = (long long)(t0 + k) * d + r;
                 if (t0 + k < t_b && i >= first && i < last) pool(win);
+                i += d;
             }
         }
     }
