@@ -385,12 +385,12 @@ __device__ __forceinline__ void s_grad_tile(const float* planes, const KRec* rec
 
 // The channels of one kernel on an S tile.  fold: the accumulators come in undefined and start at the
 // kernel's 0 - bias inside the first channel's pass (every output of the warp tile exists).
-template <int ELL>
-__device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* rec, int lane, u64 (&acc)[kR], bool fold) {
+template <int ELL, bool FOLD>
+__device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* rec, int lane, u64 (&acc)[kR]) {
     const int m = rec->m;
     const int off[4] = {2 * lane, kWarpCols + 2 * lane, 2 * kWarpCols + 2 * lane, 3 * kWarpCols + 2 * lane};
     int q = 0;
-    if (fold) {
+    if constexpr (FOLD) {
         const float nb = rec->negb;
         conv_channel<ELL, 4 * kWarpCols, false, true>(planes + rec->ch[0] * kSPlaneFloats, off, rec->w2[0], acc, 0, 0, pack2(nb, nb));
         q = 1;
@@ -487,12 +487,12 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
             }
             u64 acc[kR];
             // hard mode: the pooling masks the outputs that do not exist, so the accumulators always start inside
-            // the first channel's pass; the other modes start them at +inf where there is no output
-            const bool fold = interior || MODE == 0;
-            if (!fold) init_acc(acc, rec->negb, false, lo0, hi0, lo1, hi1);
-            if (len == 7) s_kernel_tile<7>(planes, rec, lane, acc, fold);
-            else if (len == 9) s_kernel_tile<9>(planes, rec, lane, acc, fold);
-            else s_kernel_tile<11>(planes, rec, lane, acc, fold);
+            // the first channel's pass; the other modes start them at 0 - bias, or +inf where there is no output
+            constexpr bool kFold = MODE == 0;
+            if (!kFold) init_acc(acc, rec->negb, interior, lo0, hi0, lo1, hi1);
+            if (len == 7) s_kernel_tile<7, kFold>(planes, rec, lane, acc);
+            else if (len == 9) s_kernel_tile<9, kFold>(planes, rec, lane, acc);
+            else s_kernel_tile<11, kFold>(planes, rec, lane, acc);
             if (MODE == 2) {
                 const int64_t pair = (int64_t)n * a.K + korig;
                 const float gP = __ldg(a.dfeat + 2 * pair), gM = __ldg(a.dfeat + 2 * pair + 1);
@@ -596,22 +596,12 @@ struct TShared {
 template <int ELL, int STEP, bool WIN>
 __device__ __forceinline__ bool t_channels(const float* stages, const KRec* rec, const int (&off)[4], uint32_t full0,
                                            uint32_t empty0, uint32_t& st, int lane, bool active, u64 (&acc)[kR], int gl,
-                                           int gh, bool fold) {
+                                           int gh) {
     const int m = rec->m;
     for (int q = 0; q < m; ++q) {
         const uint32_t slot = st % kTStages;
         if (q > 0 && !mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) return false;
-        if (active) {
-            bool done = false;
-            if constexpr (!WIN) {
-                if (fold && q == 0) {   // the accumulators start at 0 - bias inside the first channel's pass
-                    const float nb = rec->negb;
-                    conv_channel<ELL, STEP, false, true>(stages + slot * kTStageFloats, off, rec->w2[0], acc, 0, 0, pack2(nb, nb));
-                    done = true;
-                }
-            }
-            if (!done) conv_channel<ELL, STEP, WIN>(stages + slot * kTStageFloats, off, rec->w2[q], acc, gl, gh);
-        }
+        if (active) conv_channel<ELL, STEP, WIN>(stages + slot * kTStageFloats, off, rec->w2[q], acc, gl, gh);
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * slot);
         ++st;
@@ -657,10 +647,10 @@ __device__ __forceinline__ bool t_grad_dispatch(int len, const float* stages, co
 template <int STEP, bool WIN>
 __device__ __forceinline__ bool t_dispatch(int len, const float* stages, const KRec* rec, const int (&off)[4],
                                            uint32_t full0, uint32_t empty0, uint32_t& st, int lane, bool active,
-                                           u64 (&acc)[kR], int gl, int gh, bool fold) {
-    if (len == 7) return t_channels<7, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh, fold);
-    if (len == 9) return t_channels<9, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh, fold);
-    return t_channels<11, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh, fold);
+                                           u64 (&acc)[kR], int gl, int gh) {
+    if (len == 7) return t_channels<7, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
+    if (len == 9) return t_channels<9, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
+    return t_channels<11, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
 }
 
 template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft
@@ -824,23 +814,24 @@ __global__ void __launch_bounds__(kTBlockThreads, kTBlocksPerSM) fast_t_forward(
                 valid_rows_tc(t0 + kR * wr, r0 + lc, rec->tl, rec->rl, rec->th, rec->rh, kR, ok0, lo0, hi0);
                 valid_rows_tc(t0 + kR * wr, r0 + lc + 1, rec->tl, rec->rl, rec->th, rec->rh, kR, ok1, lo1, hi1);
             }
-            const int boxw = t_box_cols(cg);
-            int off[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                off[k] = wide ? t_wide_elem_offset(k, lc, box_rows, si.g_lo)
-                              : t_box_offset(cg, k, box_rows) + 4 * wr * boxw + lc;
+            // where rows 0..3 of the warp tile sit in a stage: the box of phase k starts k * phase floats in; an
+            // ordinary tile's warp tile starts 4 wr box rows down, a wide tile's in half lc / 256, g_lo box rows up
+            // (t_elem_offset / t_wide_elem_offset for tile rows 0..3)
+            const int boxw = wide ? kTWideCols : t_box_cols(cg);
+            const int phase = box_rows * boxw;
+            const int base = wide ? (lc >> 8) * (4 * phase) - si.g_lo * kTWideCols + (lc & (kTWideCols - 1)) : 4 * wr * boxw + lc;
+            const int off[4] = {base, base + phase, base + 2 * phase, base + 3 * phase};
             const int gl = si.g_lo, gh = si.g_hi;
             u64 acc[kR];
-            // Ordinary tiles start their accumulators inside the first channel's pass: interior warp tiles in every
-            // mode, the others in hard mode, where the pooling masks the outputs that do not exist.  Everywhere
-            // else the accumulators start at 0 - bias, or +inf where there is no output.
-            const bool fold = !wide && (interior || MODE == 0);
-            if (active && !fold) init_acc(acc, rec->negb, interior || MODE == 0, lo0, hi0, lo1, hi1);
-            if (wide) ok = t_dispatch<kTWideCols, true>(len, stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh, false);
-            else if (cg == 1) ok = t_dispatch<kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0, fold);
-            else if (cg == 2) ok = t_dispatch<2 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0, fold);
-            else ok = t_dispatch<4 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0, fold);
+            // Hard mode: every accumulator starts at 0 - bias and the pooling masks the outputs that do not exist.
+            // The other modes start at +inf where there is no output.  (Starting the accumulators inside the first
+            // channel's pass, as the small-dilation kernel does, doubles the inner-loop instances here: measured
+            // slower, the kernel then waits for instructions.)
+            if (active) init_acc(acc, rec->negb, interior || MODE == 0, lo0, hi0, lo1, hi1);
+            if (wide) ok = t_dispatch<kTWideCols, true>(len, stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
+            else if (cg == 1) ok = t_dispatch<kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
+            else if (cg == 2) ok = t_dispatch<2 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
+            else ok = t_dispatch<4 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
             if (!ok) break;
             const int64_t pair = (int64_t)n * a.K + korig;
             if (MODE == 2) {
