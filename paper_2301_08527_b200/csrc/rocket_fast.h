@@ -11,7 +11,7 @@
 // adjacent column pairs: a warp tile is 16 rows x 64 columns.
 //
 // Two regimes share the arithmetic core:
-//   S (d < split): kernels of one dilation form a bucket.  Columns of successive 16-row bands
+//   S (d < split): kernels of one dilation form a bucket.  Columns of successive bands of kRS rows
 //     are strung together into one "raster" (band-major, r-minor) and a tile is 64 consecutive
 //     raster positions, so lanes stay busy even when d < 64.  A block stages one tile of ALL
 //     channels in shared memory, then its warps pull kernels of the bucket from a shared
@@ -69,15 +69,25 @@ constexpr int kNormMaxChannels = 20;
 struct NormArgs { float mean[kNormMaxChannels], inv_std[kNormMaxChannels]; };
 
 constexpr int kSMaxChannels = 20;                                  // channels the S tile can stage
+// Output rows of a warp tile in the S regime (the band height of its rasters).  More rows per thread than in
+// the T regime: the work per (kernel, tile) grows while the per-kernel bookkeeping and the rows staged per
+// output shrink.  Measured at 60 x 20 x 50,000 (hard): 16 rows 25.7 ms, 20 rows 24.9, 22 rows 24.6, 24 to 26
+// rows 24.1 (16 warps each; 12 warps are slower at every height), 28 rows need 14 warps for the tile to fit.
+#ifndef ROCKET_S_ROWS
+#define ROCKET_S_ROWS 24
+#endif
 #ifndef ROCKET_S_THREADS
 #define ROCKET_S_THREADS 512
 #endif
+constexpr int kRS = ROCKET_S_ROWS;
+static_assert(kRS >= 8 && kRS <= 32, "the row masks of the pooling hold at most 32 rows");
+constexpr int kSRowsMax = kRS + ROCKET_MAX_LENGTH - 1;             // staged rows an S warp tile reads
 constexpr int kSThreads = ROCKET_S_THREADS, kSWarps = kSThreads / 32;   // one block per SM
-constexpr int kSPlaneFloats = kRowsMax * kWarpCols;                // one channel of an S tile
+constexpr int kSPlaneFloats = kSRowsMax * kWarpCols;               // one channel of an S tile
 
 struct SBucket {
     int32_t d, tmin, nbands, raster_len;  // raster_len = nbands * d
-    int32_t kbeg, kend, rows, pad_;       // kernels [kbeg, kend) of krec; rows = 16 + max len - 1
+    int32_t kbeg, kend, rows, pad_;       // kernels [kbeg, kend) of krec; rows = kRS + max len - 1
 };
 // One S tile: 64 raster positions from c0 of a bucket.  interior = 1 when every (row, column) of the
 // tile is an output of every kernel of the bucket (then the kernels need no range tests).

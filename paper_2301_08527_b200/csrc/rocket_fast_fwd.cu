@@ -70,9 +70,9 @@ __device__ __forceinline__ float key_float(int k) { return __int_as_float(k >= 0
 // and multiplied (the others hold no sample and are not in shared memory); gl and gh are the same
 // for the whole warp.  With FIRST the accumulators come in undefined and every one of them starts as
 // init + w[0] * x (its first product), which is bit for bit what starting at init and adding gives.
-template <int ELL, int STEP, bool WIN, bool FIRST = false>
+template <int ELL, int STEP, bool WIN, bool FIRST = false, int R = kR>
 __device__ __forceinline__ void conv_channel(const float* __restrict__ st, const int (&off)[4],
-                                             const float* __restrict__ w2, u64 (&acc)[kR], int gl = 0, int gh = 0,
+                                             const float* __restrict__ w2, u64 (&acc)[R], int gl = 0, int gh = 0,
                                              u64 init = 0ull) {
     static_assert(!(WIN && FIRST), "a windowed pass may skip an accumulator's first product");
     u64 wp[ELL + 1];
@@ -83,16 +83,16 @@ __device__ __forceinline__ void conv_channel(const float* __restrict__ st, const
         wp[j + 1] = v.y;
     }
 #pragma unroll
-    for (int g = 0; g < (kR + ELL - 1 + 3) / 4; ++g) {
+    for (int g = 0; g < (R + ELL - 1 + 3) / 4; ++g) {
         if (!WIN || (g >= gl && g < gh)) {
 #pragma unroll
-            for (int s = 4 * g; s < 4 * g + 4 && s < kR + ELL - 1; ++s) {
+            for (int s = 4 * g; s < 4 * g + 4 && s < R + ELL - 1; ++s) {
                 const float* p = st + off[s & 3] + (s >> 2) * STEP;
                 const u64 x = *reinterpret_cast<const u64*>(p);
 #pragma unroll
                 for (int j = 0; j < ELL; ++j) {
                     const int o = s - j;
-                    if (o >= 0 && o < kR) {
+                    if (o >= 0 && o < R) {
                         if (FIRST && j == 0) acc[o] = fma2_to(wp[0], x, init);
                         else fma2(acc[o], wp[j], x);
                     }
@@ -105,15 +105,17 @@ __device__ __forceinline__ void conv_channel(const float* __restrict__ st, const
 // Adds the PPV count of the thread's 2 x 16 outputs to cnt and folds their min(-z) into mn.  Outputs outside the kernel's range
 // never need a test here: their accumulators start at +inf and stay there (sign bit clear,
 // neutral for the min).
-__device__ __forceinline__ void pool_hard(const u64 (&acc)[kR], int& cnt, float& mn) {
-    unsigned signs = 0;  // one sign bit per output, shifted in from the right
+template <int R>
+__device__ __forceinline__ void pool_hard(const u64 (&acc)[R], int& cnt, float& mn) {
+    unsigned signs = 0;  // one sign bit per output, shifted in from the right (counted every 16 rows)
 #pragma unroll
-    for (int o = 0; o < kR; ++o) {
+    for (int o = 0; o < R; ++o) {
         float a, b;
         unpack2(acc[o], a, b);
         signs = __funnelshift_l(__float_as_uint(a), signs, 1);
         signs = __funnelshift_l(__float_as_uint(b), signs, 1);
         mn = min3(mn, a, b);
+        if ((o & 15) == 15 && o + 1 < R) { cnt += __popc(signs); signs = 0; }
     }
     cnt += __popc(signs);
 }
@@ -121,11 +123,12 @@ __device__ __forceinline__ void pool_hard(const u64 (&acc)[kR], int& cnt, float&
 // The same for a warp tile with outputs that do not exist: m0 / m1 hold one bit per row of the thread's two
 // columns (bit o set: row o is an output); the others are replaced by +inf on the way (sign bit clear, neutral
 // for the min), so the accumulators may hold anything there.
-__device__ __forceinline__ void pool_hard_masked(const u64 (&acc)[kR], unsigned m0, unsigned m1, int& cnt, float& mn) {
+template <int R>
+__device__ __forceinline__ void pool_hard_masked(const u64 (&acc)[R], unsigned m0, unsigned m1, int& cnt, float& mn) {
     const float inf = __int_as_float(0x7f800000);
     unsigned signs = 0;
 #pragma unroll
-    for (int o = 0; o < kR; ++o) {
+    for (int o = 0; o < R; ++o) {
         float a, b;
         unpack2(acc[o], a, b);
         a = (m0 & (1u << o)) ? a : inf;
@@ -133,22 +136,24 @@ __device__ __forceinline__ void pool_hard_masked(const u64 (&acc)[kR], unsigned 
         signs = __funnelshift_l(__float_as_uint(a), signs, 1);
         signs = __funnelshift_l(__float_as_uint(b), signs, 1);
         mn = min3(mn, a, b);
+        if ((o & 15) == 15 && o + 1 < R) { cnt += __popc(signs); signs = 0; }
     }
     cnt += __popc(signs);
 }
-// Bit o set for lo <= o < hi (0 <= lo, hi <= 16).
+// Bit o set for lo <= o < hi (0 <= lo, hi <= 31).
 __device__ __forceinline__ unsigned row_mask(int lo, int hi) { return hi > lo ? ((1u << hi) - 1u) & ~((1u << lo) - 1u) : 0u; }
 
 // Accumulators of a tile: 0 - bias where the output exists, +inf elsewhere.
-__device__ __forceinline__ void init_acc(u64 (&acc)[kR], float negb, bool interior, int lo0, int hi0, int lo1, int hi1) {
+template <int R>
+__device__ __forceinline__ void init_acc(u64 (&acc)[R], float negb, bool interior, int lo0, int hi0, int lo1, int hi1) {
     if (interior) {
         const u64 v = pack2(negb, negb);
 #pragma unroll
-        for (int o = 0; o < kR; ++o) acc[o] = v;
+        for (int o = 0; o < R; ++o) acc[o] = v;
     } else {
         const float inf = __int_as_float(0x7f800000);
 #pragma unroll
-        for (int o = 0; o < kR; ++o) acc[o] = pack2((o >= lo0 && o < hi0) ? negb : inf, (o >= lo1 && o < hi1) ? negb : inf);
+        for (int o = 0; o < R; ++o) acc[o] = pack2((o >= lo0 && o < hi0) ? negb : inf, (o >= lo1 && o < hi1) ? negb : inf);
     }
 }
 
@@ -185,14 +190,15 @@ constexpr float kSoftFixedScale = 1073741824.0f;  // 2^30: soft sums travel as f
 // step the index distance between rows.  The warp's sum is added to ws[2 * pair] as a fixed-point
 // integer and (max key, INT_MAX - index) is folded into ws[2 * pair + 1] with one 64-bit atomic max:
 // both are exact and order-free, so results are run-to-run identical.
-__device__ __forceinline__ void pool_publish_soft(unsigned long long* __restrict__ ws, int64_t pair, const u64 (&acc)[kR],
+template <int R>
+__device__ __forceinline__ void pool_publish_soft(unsigned long long* __restrict__ ws, int64_t pair, const u64 (&acc)[R],
                                                   float c1, float c0, bool interior, int lo0, int hi0, int lo1, int hi1,
                                                   int base0, int base1, int step, int lane) {
     const u64 c1p = pack2(c1, c1), c0p = pack2(c0, c0), one = pack2(1.0f, 1.0f);
     u64 hs = pack2(0.0f, 0.0f);
     float mn = __int_as_float(0x7f800000);
 #pragma unroll
-    for (int o = 0; o < kR; ++o) {
+    for (int o = 0; o < R; ++o) {
         u64 t = c0p;
         fma2(t, acc[o], c1p);
         float ta, tb, a, b;
@@ -218,7 +224,7 @@ __device__ __forceinline__ void pool_publish_soft(unsigned long long* __restrict
     int idx = INT_MAX;
     if (key == wkey) {
 #pragma unroll
-        for (int o = kR - 1; o >= 0; --o) {
+        for (int o = R - 1; o >= 0; --o) {
             float a, b;
             unpack2(acc[o], a, b);
             if (b == mn) idx = min(idx, base1 + o * step);
@@ -244,13 +250,14 @@ __device__ __forceinline__ u64 mul2(u64 a, u64 b) {
 //   gz = gPs * h (1 - h) + gM [output index == argmax],  h = 1 / (1 + 2^(c1 * acc + c0)),
 // zero where the output does not exist, and returns the thread's sum of gz (its share of db).
 // oA0 / oA1: the row of the thread's first / second column that is the argmax, or -1.
-__device__ __forceinline__ float make_gz(u64 (&acc)[kR], float c1, float c0, float gPs, float gM, bool interior, int lo0,
+template <int R>
+__device__ __forceinline__ float make_gz(u64 (&acc)[R], float c1, float c0, float gPs, float gM, bool interior, int lo0,
                                          int hi0, int lo1, int hi1, int oA0, int oA1) {
     const u64 c1p = pack2(c1, c1), c0p = pack2(c0, c0), one = pack2(1.0f, 1.0f), neg1 = pack2(-1.0f, -1.0f);
     const u64 gp = pack2(gPs, gPs);
     u64 sum = pack2(0.0f, 0.0f);
 #pragma unroll
-    for (int o = 0; o < kR; ++o) {
+    for (int o = 0; o < R; ++o) {
         u64 t = c0p;
         fma2(t, acc[o], c1p);
         float ta, tb;
@@ -280,20 +287,20 @@ __device__ __forceinline__ float make_gz(u64 (&acc)[kR], float c1, float c0, flo
 
 // Backward, second half, one channel of one warp tile: dw[j] += gz[o] * x[o + j] for the thread's
 // column pair (same traversal as conv_channel with the roles of weights and accumulators swapped).
-template <int ELL, int STEP, bool WIN>
-__device__ __forceinline__ void grad_channel(const float* __restrict__ st, const int (&off)[4], const u64 (&gz)[kR],
+template <int ELL, int STEP, bool WIN, int R = kR>
+__device__ __forceinline__ void grad_channel(const float* __restrict__ st, const int (&off)[4], const u64 (&gz)[R],
                                              u64 (&dw)[ELL], int gl = 0, int gh = 0) {
 #pragma unroll
-    for (int g = 0; g < (kR + ELL - 1 + 3) / 4; ++g) {
+    for (int g = 0; g < (R + ELL - 1 + 3) / 4; ++g) {
         if (!WIN || (g >= gl && g < gh)) {
 #pragma unroll
-            for (int s = 4 * g; s < 4 * g + 4 && s < kR + ELL - 1; ++s) {
+            for (int s = 4 * g; s < 4 * g + 4 && s < R + ELL - 1; ++s) {
                 const float* p = st + off[s & 3] + (s >> 2) * STEP;
                 const u64 x = *reinterpret_cast<const u64*>(p);
 #pragma unroll
                 for (int j = 0; j < ELL; ++j) {
                     const int o = s - j;
-                    if (o >= 0 && o < kR) fma2(dw[j], gz[o], x);
+                    if (o >= 0 && o < R) fma2(dw[j], gz[o], x);
                 }
             }
         }
@@ -370,7 +377,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 
 // Backward second half for one kernel on an S tile: per channel, dW sums of the warp tile.
 template <int ELL>
-__device__ __forceinline__ void s_grad_tile(const float* planes, const KRec* rec, int lane, const u64 (&gz)[kR],
+__device__ __forceinline__ void s_grad_tile(const float* planes, const KRec* rec, int lane, const u64 (&gz)[kRS],
                                             long long* accfix, double scale) {
     const int m = rec->m;
     const int off[4] = {2 * lane, kWarpCols + 2 * lane, 2 * kWarpCols + 2 * lane, 3 * kWarpCols + 2 * lane};
@@ -378,7 +385,7 @@ __device__ __forceinline__ void s_grad_tile(const float* planes, const KRec* rec
         u64 dw[ELL];
 #pragma unroll
         for (int j = 0; j < ELL; ++j) dw[j] = 0ull;
-        grad_channel<ELL, 4 * kWarpCols, false>(planes + rec->ch[q] * kSPlaneFloats, off, gz, dw);
+        grad_channel<ELL, 4 * kWarpCols, false, kRS>(planes + rec->ch[q] * kSPlaneFloats, off, gz, dw);
         reduce_publish_dw<ELL>(dw, accfix + rec->woff + q * ELL, scale, lane);
     }
 }
@@ -386,17 +393,17 @@ __device__ __forceinline__ void s_grad_tile(const float* planes, const KRec* rec
 // The channels of one kernel on an S tile.  fold: the accumulators come in undefined and start at the
 // kernel's 0 - bias inside the first channel's pass (every output of the warp tile exists).
 template <int ELL, bool FOLD>
-__device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* rec, int lane, u64 (&acc)[kR]) {
+__device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* rec, int lane, u64 (&acc)[kRS]) {
     const int m = rec->m;
     const int off[4] = {2 * lane, kWarpCols + 2 * lane, 2 * kWarpCols + 2 * lane, 3 * kWarpCols + 2 * lane};
     int q = 0;
     if constexpr (FOLD) {
         const float nb = rec->negb;
-        conv_channel<ELL, 4 * kWarpCols, false, true>(planes + rec->ch[0] * kSPlaneFloats, off, rec->w2[0], acc, 0, 0, pack2(nb, nb));
+        conv_channel<ELL, 4 * kWarpCols, false, true, kRS>(planes + rec->ch[0] * kSPlaneFloats, off, rec->w2[0], acc, 0, 0, pack2(nb, nb));
         q = 1;
     }
     for (; q < m; ++q)
-        conv_channel<ELL, 4 * kWarpCols, false>(planes + rec->ch[q] * kSPlaneFloats, off, rec->w2[q], acc);
+        conv_channel<ELL, 4 * kWarpCols, false, false, kRS>(planes + rec->ch[q] * kSPlaneFloats, off, rec->w2[q], acc);
 }
 
 template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft
@@ -448,7 +455,7 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
         const bool ok0 = cg0 < b.raster_len, ok1 = cg0 + 1 < b.raster_len;
         const int band0 = cg0 / d, c0 = cg0 - band0 * d;          // (first A-row, residue) of the two columns
         const int band1 = c0 + 1 < d ? band0 : band0 + 1, c1 = c0 + 1 < d ? c0 + 1 : 0;
-        const int trow0 = b.tmin + band0 * kR, trow1 = b.tmin + band1 * kR;
+        const int trow0 = b.tmin + band0 * kRS, trow1 = b.tmin + band1 * kRS;
         if (threadIdx.x == 0) s_next = b.kbeg;
         cp_async_wait<0>();
         __syncthreads();
@@ -478,14 +485,14 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
             const KRec* rec = myrec + cur;
             const int len = rec->len, korig = rec->k;
             // on an interior tile (the plan's flag) every output exists for every kernel of the bucket
-            int lo0 = 0, hi0 = kR, lo1 = 0, hi1 = kR;
+            int lo0 = 0, hi0 = kRS, lo1 = 0, hi1 = kRS;
             bool interior = tile_interior;
             if (!tile_interior) {
-                valid_rows_tc(trow0, c0, rec->tl, rec->rl, rec->th, rec->rh, kR, ok0, lo0, hi0);
-                valid_rows_tc(trow1, c1, rec->tl, rec->rl, rec->th, rec->rh, kR, ok1, lo1, hi1);
-                interior = __all_sync(kFull, lo0 == 0 && lo1 == 0 && hi0 == kR && hi1 == kR);
+                valid_rows_tc(trow0, c0, rec->tl, rec->rl, rec->th, rec->rh, kRS, ok0, lo0, hi0);
+                valid_rows_tc(trow1, c1, rec->tl, rec->rl, rec->th, rec->rh, kRS, ok1, lo1, hi1);
+                interior = __all_sync(kFull, lo0 == 0 && lo1 == 0 && hi0 == kRS && hi1 == kRS);
             }
-            u64 acc[kR];
+            u64 acc[kRS];
             // hard mode: the pooling masks the outputs that do not exist, so the accumulators always start inside
             // the first channel's pass; the other modes start them at 0 - bias, or +inf where there is no output
             constexpr bool kFold = MODE == 0;
@@ -499,8 +506,8 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
                 const int uA = __ldg(a.argmax + pair) - rec->p;
                 int tA = uA / d, cA = uA - tA * d;                        // floor division: uA >= -p may be negative
                 if (cA < 0) { cA += d; --tA; }
-                const int oA0 = (ok0 && c0 == cA && tA >= trow0 && tA < trow0 + kR) ? tA - trow0 : -1;
-                const int oA1 = (ok1 && c1 == cA && tA >= trow1 && tA < trow1 + kR) ? tA - trow1 : -1;
+                const int oA0 = (ok0 && c0 == cA && tA >= trow0 && tA < trow0 + kRS) ? tA - trow0 : -1;
+                const int oA1 = (ok1 && c1 == cA && tA >= trow1 && tA < trow1 + kRS) ? tA - trow1 : -1;
                 float dbs = make_gz(acc, a.c1, a.c0, gP * a.lambda / (float)rec->nout, gM, interior, lo0, hi0, lo1, hi1, oA0, oA1);
 #pragma unroll
                 for (int sh = 16; sh > 0; sh >>= 1) dbs += __shfl_xor_sync(kFull, dbs, sh);

@@ -37,7 +37,7 @@ ROCKET_HD void valid_rows_tc(int t_row0, int c, int tl, int rl, int th, int rh, 
 // S regime: the u of the first output row of raster column cg of a bucket.
 ROCKET_HD int s_column_u0(const SBucket& b, int cg) {
     const int band = cg / b.d, r = cg - band * b.d;
-    return (b.tmin + band * kR) * b.d + r;
+    return (b.tmin + band * kRS) * b.d + r;
 }
 
 // T regime.  A tile starts at A-row t0 and residue r0 (a multiple of 64).  Row s of the tile

@@ -84,9 +84,9 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         }
         b.kend = (int32_t)out.krec.size();
         b.tmin = (int32_t)tmin;
-        b.nbands = (int32_t)((tmax - tmin + 1 + kR - 1) / kR);
+        b.nbands = (int32_t)((tmax - tmin + 1 + kRS - 1) / kRS);
         b.raster_len = b.nbands * d;
-        b.rows = kR + maxlen - 1;
+        b.rows = kRS + maxlen - 1;
         const int bi = (int)out.sb.size();
         out.sb.push_back(b);
         // a tile is interior when its 64 raster positions exist and the u of every (row, column) lies inside
@@ -100,7 +100,7 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
             bool interior = c0 + kWarpCols <= b.raster_len;
             for (int c = c0; interior && c < c0 + kWarpCols; ++c) {
                 const int64_t u0 = s_column_u0(b, c);
-                interior = u0 >= lo_max && u0 + (int64_t)(kR - 1) * d < hi_min;
+                interior = u0 >= lo_max && u0 + (int64_t)(kRS - 1) * d < hi_min;
             }
             s_cost.push_back({work + 0.3 * hp.C * b.rows, (int)out.sitems.size()});
             out.sitems.push_back({bi, c0, interior ? 1 : 0, 0});

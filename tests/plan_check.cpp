@@ -56,7 +56,7 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
 
     for (const SItem& it : plan.sitems) {
         const SBucket& b = plan.sb[it.bucket];
-        REQUIRE(b.rows <= kRowsMax && b.d < plan.split && it.c0 % kWarpCols == 0, "S bucket shape");
+        REQUIRE(b.rows <= kSRowsMax && b.d < plan.split && it.c0 % kWarpCols == 0, "S bucket shape");
         bool all_full = true;
         for (int col = 0; col < kWarpCols; ++col) {
             const int cg = it.c0 + col;
@@ -64,13 +64,13 @@ static int check(uint64_t seed, int K, int C, int L, int split, const HostParams
             const int u0 = s_column_u0(b, cg);
             for (int kk = b.kbeg; kk < b.kend; ++kk) {
                 const KRec& f = plan.krec[kk];
-                REQUIRE(f.d == b.d && kR + f.len - 1 <= b.rows, "S kernel in wrong bucket");
+                REQUIRE(f.d == b.d && kRS + f.len - 1 <= b.rows, "S kernel in wrong bucket");
                 int o_lo, o_hi, q_lo, q_hi;
-                valid_rows(u0, b.d, f.lo_u, f.hi_u, kR, col_ok, q_lo, q_hi);
+                valid_rows(u0, b.d, f.lo_u, f.hi_u, kRS, col_ok, q_lo, q_hi);
                 const int band = cg / b.d;
-                valid_rows_tc(b.tmin + band * kR, cg - band * b.d, f.tl, f.rl, f.th, f.rh, kR, col_ok, o_lo, o_hi);
+                valid_rows_tc(b.tmin + band * kRS, cg - band * b.d, f.tl, f.rl, f.th, f.rh, kRS, col_ok, o_lo, o_hi);
                 REQUIRE((o_lo >= o_hi && q_lo >= q_hi) || (o_lo == q_lo && o_hi == q_hi), "S row range: the two forms disagree");
-                all_full = all_full && o_lo == 0 && o_hi == kR;
+                all_full = all_full && o_lo == 0 && o_hi == kRS;
                 for (int o = o_lo; o < o_hi; ++o) {
                     const int64_t i = (int64_t)u0 + (int64_t)o * b.d + f.p;
                     REQUIRE(i >= 0 && i < f.nout, "S output out of range");
