@@ -44,7 +44,10 @@ namespace fast {
 constexpr int kR = 16;                                             // output rows of a warp tile
 constexpr int kWarpCols = 64;                                      // columns of a warp tile (2 per lane)
 constexpr int kRowsMax = kR + ROCKET_MAX_LENGTH - 1;               // staged rows a warp tile reads
-constexpr int kSplitDefault = 64;                                  // S below, T at or above
+#ifndef ROCKET_SPLIT
+#define ROCKET_SPLIT 64
+#endif
+constexpr int kSplitDefault = ROCKET_SPLIT;                        // S below, T at or above
 constexpr int kTMinDilation = 64;                                  // a T tile needs 64 residues in one band
 
 // ---- kernel record: one fast kernel as the device reads it (header + duplicated weights) ----
