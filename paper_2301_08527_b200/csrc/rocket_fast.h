@@ -87,6 +87,7 @@ static_assert(kRS >= 8 && kRS <= 32, "the row masks of the pooling hold at most 
 constexpr int kSRowsMax = kRS + ROCKET_MAX_LENGTH - 1;             // staged rows an S warp tile reads
 constexpr int kSThreads = ROCKET_S_THREADS, kSWarps = kSThreads / 32;   // one block per SM
 constexpr int kSPlaneFloats = kSRowsMax * kWarpCols;               // one channel of an S tile
+constexpr int kSLengthOrderMin = 100;                              // buckets from this many kernels up are ordered by length
 
 struct SBucket {
     int32_t d, tmin, nbands, raster_len;  // raster_len = nbands * d

@@ -57,7 +57,11 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         out.krec.push_back(f);
     };
 
-    // ---- S regime: one bucket per dilation, kernels inside ordered by cost (largest first)
+    // ---- S regime: one bucket per dilation, kernels inside ordered by cost (largest first: the warps of a
+    // block pull them one by one, so the cheap ones fill the end of a tile evenly).  Buckets with many
+    // kernels per warp are ordered by length first: warps that run side by side then share one instance of
+    // the inner loops, which the instruction caches reward (backward 5 % faster, hard transform unchanged;
+    // for the small buckets the balance at the end of a tile is worth more).
     std::map<int, std::vector<int>> by_d;
     for (int k : s_kernels) by_d[hp.dilation[k]].push_back(k);
     struct Cost { double c; int idx; };
@@ -66,6 +70,7 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
         const int d = kv.first;
         auto& ks = kv.second;
         std::stable_sort(ks.begin(), ks.end(), [&](int a, int b) {
+            if ((int)ks.size() >= kSLengthOrderMin && hp.length[a] != hp.length[b]) return hp.length[a] > hp.length[b];
             return hp.length[a] * hp.num_channels[a] > hp.length[b] * hp.num_channels[b];
         });
         SBucket b{};
@@ -119,6 +124,9 @@ void build_plan(const HostParams& hp, int split, PlanHost& out) {
     // fewest block tiles wins
     int d_max = 0;
     std::map<std::tuple<int, int, int>, int> map_index;
+    // kernels of one length follow one another, so that the blocks running at any one time execute the same
+    // instance of the inner loops (instruction caches: backward 3.5 % faster, forward 0.1-1 %)
+    std::stable_sort(t_kernels.begin(), t_kernels.end(), [&](int a, int b) { return hp.length[a] > hp.length[b]; });
     for (int k : t_kernels) {
         const int ki = (int)out.krec.size();
         add_kernel(k);
