@@ -33,6 +33,7 @@ TRAIN = dict(N=32, C=20, L=50000, K=10000)           # soft forward + backward s
 PARAM_SEED, DATA_SEED, GRAD_SEED = 8527, 2301, 527
 LAMBDA, SHIFT = 10.0, 3.0
 
+MINI_FEATURES = 9996          # MINIROCKET's default 10,000 rounded down to a multiple of its 84 kernels
 # DRAM bytes (read + write) of one launch of either fused kernel, from the committed ncu capture (profiles/),
 # per launch = one chunk of 12 examples.  The figures belong to one state of the kernel sources: they are
 # reported only while the digest of those sources still equals NCU_SOURCES_DIGEST, and as null otherwise.
@@ -215,8 +216,9 @@ def main():
                     "calls each) on rank 0 instead of its time-boxed default (12 points, one timed call each)")
     ap.add_argument("--skip-sweep", action="store_true", help="skip the throughput sweep")
     ap.add_argument("--small", action="store_true", help="profiling case: N=12 examples, one launch of either fused kernel")
-    ap.add_argument("--profile-pass", choices=["soft", "backward"], default=None,
-                    help="profiling case: run only that pass of config 3 on 12 examples, three times, and exit")
+    ap.add_argument("--profile-pass", choices=["soft", "backward", "minirocket"], default=None,
+                    help="profiling case: run only that pass (config 3's soft forward or backward, or the MINIROCKET "
+                         "transform with 9,996 features) on 12 examples, three times, and exit")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -265,6 +267,19 @@ def main():
         # one launch of either fused kernel per call: the case the ncu captures of the soft forward and
         # of the backward use
         Xs = X[:12].contiguous()
+        if args.profile_pass == "minirocket":
+            mr = rk.MiniRocket.create(PARAM_SEED, w["C"], w["L"], MINI_FEATURES)
+            mr.fit(X_host[:12].numpy())
+            mfeat = mr.transform(Xs)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(2):
+                mr.transform(Xs, out=mfeat)
+            e1.record()
+            torch.cuda.synchronize()
+            print(json.dumps({"pass": "minirocket", "shape": "N=12 x C=%d x L=%d, %d features" % (w["C"], w["L"], MINI_FEATURES),
+                              "ms": e0.elapsed_time(e1) / 2}))
+            return
         sfeat, arg = rk.rocket_transform_soft(params, Xs, LAMBDA, SHIFT)
         g = torch.from_numpy(normal_array(GRAD_SEED, (12, 2 * w["K"]))).cuda()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -423,7 +438,19 @@ def main():
         s_pred, _ = time_steps(lambda: rk.rocket_ridge_predict(feat, wr, br, out=yhat), 5, 3)
         s_pred /= 5
         del Fr
+        # MINIROCKET on the same batch (Section 2; Section 6, last sentence): host fit, then the fused transform
+        mr = rk.MiniRocket.create(PARAM_SEED, w["C"], w["L"], MINI_FEATURES)
+        t0 = time.perf_counter()
+        mr.fit(X_host.numpy()[:16])
+        s_mfit = time.perf_counter() - t0
+        mfeat = mr.transform(X)
+        s_mini, _ = time_steps(lambda: mr.transform(X, out=mfeat), psteps, 3)
+        s_mini = max_over(s_mini) / psteps
+        mr.close()
+        del mfeat
         passes = {
+            "minirocket": {"shape": "N=%d x C=%d x L=%d, %d features" % (w["N"], w["C"], w["L"], MINI_FEATURES),
+                           "examples_per_s": world * w["N"] / s_mini, "ms": 1e3 * s_mini, "host_fit_s": s_mfit},
             "ridge": {"fit_ms": 1e3 * s_fit, "fit_shape": "677 examples x %d features, alpha=1" % (2 * w["K"]),
                       "predict_ms": 1e3 * s_pred, "predict_shape": "%d examples x %d features" % (w["N"], 2 * w["K"])},
             "hard_u8": {"shape": "N=%d x C=%d x L=%d uint8, K=%d" % (w["N"], w["C"], w["L"], w["K"]),

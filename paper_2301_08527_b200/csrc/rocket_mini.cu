@@ -7,22 +7,25 @@
 //                every other (dilation, kernel) combination, a random channel subset per combination
 //   fit          rocket_mini_fit, on the host (a one-off over one training example per combination): the bias of
 //                a feature is a quantile of the combination's convolution output on that example
-//   transform    rocket_mini_transform, one fused kernel: per (example, combination) the channels are summed, the
-//                nine-tap dilated convolution runs on a register window that slides down a column of the
-//                dilated view, and every output is compared with the combination's biases on the fly, so the
-//                convolution outputs never reach memory; feature = count / number of outputs (Eq. 1-2 against
-//                the bias)
+//   transform    rocket_mini_transform, one fused kernel: per (example, combination) the channels are summed into
+//                a shared-memory tile of the dilated view, the nine-tap dilated convolution runs on a register
+//                window that slides down a column of the tile, and every output is compared with the
+//                combination's biases on the fly, so the convolution outputs never reach memory; feature =
+//                count / number of outputs (Eq. 1-2 against the bias)
 //
 // The kernel weights take two values, so every product is one fused multiply-add with -1 or 2: on this
 // hardware an addition and a fused multiply-add take the same issue slot, and the additions-only form that
 // speeds the method up on a CPU brings nothing here.  The bound of the kernel is the traffic from L2: every
 // combination reads its channels once.
 #include <algorithm>
+#include <array>
 #include <cmath>
+#include <map>
 #include <mutex>
 #include <new>
 #include <numeric>
 #include <thread>
+#include <type_traits>
 #include <vector>
 
 #include "rocket_internal.h"
@@ -30,10 +33,15 @@
 namespace {
 
 constexpr int kKernels = 84, kLen = 9;
-constexpr int kMaxFeaturesPerItem = 16;
+constexpr int kMaxFeaturesPerItem = 8;      // a combination with more features becomes several items
 constexpr int kThreads = 256;
-constexpr int kSmallDilation = 32;     // below: consecutive outputs from a staged run of samples; from here on: column walks
-constexpr int kChunk = 4096;           // outputs per staged run
+#ifndef ROCKET_MINI_TILE
+#define ROCKET_MINI_TILE (16 * 1024)
+#endif
+constexpr int kTileSamples = ROCKET_MINI_TILE;
+#ifndef ROCKET_MINI_BLOCKS
+#define ROCKET_MINI_BLOCKS 3
+#endif   // channel-summed samples a block stages at a time (64 KB of shared memory)
 constexpr uint64_t kGolden = 0x9E3779B97F4A7C15ull;
 constexpr uint64_t kStreamBase = 1ull << 32;
 constexpr double kInvGoldenRatio = 0.6180339887498949;
@@ -50,124 +58,227 @@ inline double draw_uniform(uint64_t seed, uint64_t stream, uint64_t slot) {
     return static_cast<double>(draw_u64(seed, stream, slot) >> 11) * 0x1.0p-53;
 }
 
-// One unit of device work: a combination, or a slice of at most 16 of its features.
+// One unit of device work: a combination, or a slice of at most 8 of its features, with the tiling of the
+// dilated view the kernel uses for its dilation (chosen on the host, choose_tiling).
 struct MiniItem {
     int32_t d, padded, m, f0, nf;
     int32_t tap[3];
     int32_t ch[kLen];
-    int32_t pad_[3];
+    int32_t width, seg_rows, segs;   // columns of a tile (= its pitch), rows a thread walks, such runs per tile
 };
 static_assert(sizeof(MiniItem) == 80, "MiniItem layout");
 
-__global__ void __launch_bounds__(kThreads)
+// Sample k of a channel row through the read-only path: at a constant byte offset from the row's first sample
+// (STRIDE samples apart), or, with a run-time stride, at an address formed by one widening multiply-add.
+template <int STRIDE>
+__device__ __forceinline__ float load_at(const float* __restrict__ x0, int k, int stride) {
+    float v;
+    if constexpr (STRIDE != 0) {
+        switch (k) {   // k is a constant after unrolling; the offset must be an immediate
+            case 0: asm("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(x0)); break;
+            case 1: asm("ld.global.nc.f32 %0, [%1+%2];" : "=f"(v) : "l"(x0), "n"(4 * STRIDE)); break;
+            case 2: asm("ld.global.nc.f32 %0, [%1+%2];" : "=f"(v) : "l"(x0), "n"(8 * STRIDE)); break;
+            case 3: asm("ld.global.nc.f32 %0, [%1+%2];" : "=f"(v) : "l"(x0), "n"(12 * STRIDE)); break;
+            case 4: asm("ld.global.nc.f32 %0, [%1+%2];" : "=f"(v) : "l"(x0), "n"(16 * STRIDE)); break;
+            case 5: asm("ld.global.nc.f32 %0, [%1+%2];" : "=f"(v) : "l"(x0), "n"(20 * STRIDE)); break;
+            case 6: asm("ld.global.nc.f32 %0, [%1+%2];" : "=f"(v) : "l"(x0), "n"(24 * STRIDE)); break;
+            default: asm("ld.global.nc.f32 %0, [%1+%2];" : "=f"(v) : "l"(x0), "n"(28 * STRIDE)); break;
+        }
+    } else {
+        const float* p;
+        asm("mad.wide.s32 %0, %1, 4, %2;" : "=l"(p) : "r"(k * stride), "l"(x0));
+        asm("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    }
+    return v;
+}
+
+// One output of the convolution from the nine window entries (the oldest sits in slot S0; taps are taken in
+// the order 0..8 whatever the slot), compared with the first 4 NG biases of the item (Eq. 1 against the bias).
+template <int S0, int NG>
+__device__ __forceinline__ void mini_pool(const float (&win)[kLen], const float (&w)[kLen],
+                                          const float (&b)[kMaxFeaturesPerItem], int (&cnt)[kMaxFeaturesPerItem]) {
+    float z = 0.0f;
+#pragma unroll
+    for (int j = 0; j < kLen; ++j) z = fmaf(w[j], win[(S0 + j) % kLen], z);
+    // Eq. 1 against every bias: one compare and one predicated add each
+#pragma unroll
+    for (int f = 0; f < 4 * NG; ++f)
+        asm("{ .reg .pred p; setp.gt.f32 p, %1, %2; @p add.s32 %0, %0, 1; }" : "+r"(cnt[f]) : "f"(z), "f"(b[f]));
+}
+
+// Steps K .. 8 of a group of nine outputs: the next row's sample enters the slot the oldest one leaves, so
+// the window never moves between registers.  GUARD: the run may end inside the group.
+template <int K, bool GUARD, int NG>
+__device__ __forceinline__ void mini_steps(const float*& p, int pitch, int left, float (&win)[kLen], const float (&w)[kLen],
+                                           const float (&b)[kMaxFeaturesPerItem], int (&cnt)[kMaxFeaturesPerItem]) {
+    if constexpr (K < kLen) {
+        if (!GUARD || K < left) {
+            win[(K + kLen - 1) % kLen] = *p;
+            p += pitch;
+            mini_pool<K, NG>(win, w, b, cnt);
+        }
+        mini_steps<K + 1, GUARD, NG>(p, pitch, left, win, w, b, cnt);
+    }
+}
+
+// The walks over one staged tile: thread u of cols * segs takes column u % cols over run u / cols.
+template <int NG>
+__device__ __forceinline__ void mini_walk_tile(const float* s_x, int P, int cols, int rows, int seg_rows, int ta, int ca,
+                                               int d, int t_min, int last, const float (&w)[kLen],
+                                               const float (&b)[kMaxFeaturesPerItem], int (&cnt)[kMaxFeaturesPerItem]) {
+    const int segs = (rows + seg_rows - 1) / seg_rows;
+    for (int u = threadIdx.x; u < cols * segs; u += kThreads) {
+        const int seg = u / cols, c = u - seg * cols;
+        // rows of this run that are outputs: t >= t_min and t d + column < last
+        const int col = ca + c;
+        const int t_end = last > col ? (last - col + d - 1) / d : 0;
+        const int t_lo = max(ta + seg * seg_rows, t_min);
+        const int t_hi = min(min(ta + rows, ta + (seg + 1) * seg_rows), t_end);
+        int left = t_hi - t_lo;
+        if (left <= 0) continue;
+        // the window of output row t holds rows t - 4 .. t + 4; staged row 0 is row ta - 4
+        const float* p = s_x + (t_lo - ta) * P + c;
+        float win[kLen];
+#pragma unroll
+        for (int j = 0; j < kLen - 1; ++j) { win[j] = *p; p += P; }
+        for (; left >= kLen; left -= kLen) mini_steps<0, false, NG>(p, P, left, win, w, b, cnt);
+        mini_steps<0, true, NG>(p, P, left, win, w, b, cnt);
+    }
+}
+
+// One block per (example, item).  The series is seen as rows of d samples (A[t][c] = x[t d + c]); a tile of it -
+// rows [ta - 4, ta + rows + 4) of `width` columns, channels already summed, zeros outside the series - is
+// staged in shared memory, then every thread walks down one column over a run of seg_rows rows with the nine
+// taps in registers: one shared-memory load, nine multiply-adds and the bias compares per output.
+__global__ void __launch_bounds__(kThreads, ROCKET_MINI_BLOCKS)
 mini_transform_kernel(const float* __restrict__ X, int C, int L, const MiniItem* __restrict__ items, int n_items,
                       const float* __restrict__ bias, float* __restrict__ feat, int F) {
+    extern __shared__ float s_x[];
     __shared__ int s_cnt[kMaxFeaturesPerItem];
-    __shared__ float s_x[kChunk + 8 * kSmallDilation];
+    __shared__ int s_choff[kLen];
     const int n = blockIdx.x / n_items;
-    const MiniItem it = items[blockIdx.x - n * n_items];
+    const MiniItem* __restrict__ item = items + (blockIdx.x - n * n_items);
+    const MiniItem it = *item;
     const float* __restrict__ Xn = X + (size_t)n * C * L;
-    if (threadIdx.x < kMaxFeaturesPerItem) s_cnt[threadIdx.x] = 0;
-    __syncthreads();
-    const int d = it.d, m = it.m;
+    const int tid = threadIdx.x;
+    if (tid < kMaxFeaturesPerItem) s_cnt[tid] = 0;
+    if (tid < kLen) s_choff[tid] = __ldg(item->ch + (tid < it.m ? tid : 0)) * L;     // C L < 2^31 (checked at creation)
+    const int d = it.d, m = it.m, nf = it.nf;
     const int first = it.padded ? 0 : 4 * d, last = it.padded ? L : L - 4 * d;
     float w[kLen];
 #pragma unroll
     for (int j = 0; j < kLen; ++j) w[j] = (j == it.tap[0] || j == it.tap[1] || j == it.tap[2]) ? 2.0f : -1.0f;
     float b[kMaxFeaturesPerItem];
 #pragma unroll
-    for (int f = 0; f < kMaxFeaturesPerItem; ++f) b[f] = f < it.nf ? __ldg(bias + it.f0 + f) : __int_as_float(0x7f800000);
+    for (int f = 0; f < kMaxFeaturesPerItem; ++f) b[f] = f < nf ? __ldg(bias + it.f0 + f) : __int_as_float(0x7f800000);
     int cnt[kMaxFeaturesPerItem];
 #pragma unroll
     for (int f = 0; f < kMaxFeaturesPerItem; ++f) cnt[f] = 0;
 
-    // the series seen as rows of d samples: a thread walks down one column over a run of rows
-    const int T = (L + d - 1) / d;
-    const int nseg = max(1, min(T, (1024 + d - 1) / d));
-    const int rows_per_seg = (T + nseg - 1) / nseg;
-    const int n_units = d * nseg;
-    // channel rows of this example (unused entries repeat the first: their loads are predicated off)
-    const float* __restrict__ chan[kLen];
+    const int T = (L + d - 1) / d;                       // rows of the dilated view
+    const int P = it.width, seg_rows = it.seg_rows;      // P: columns of a tile and its pitch in shared memory
+    const int tile_rows = seg_rows * it.segs;
+    const bool whole_rows = P == d;                      // a tile spans whole rows: its samples are one contiguous run
+    const int t_min = it.padded ? 0 : 4;                 // rows below hold no output of an unpadded combination
+    const int groups = (nf + 3) / 4;
+
+    // NK staged samples per thread at a time: position base + k * stride goes to slot + k * slot_stride.  The
+    // channels are taken two at a time, so that 2 NK loads are in flight per thread.  CHECK: a sample may lie
+    // beyond the series (then it is zero).  STRIDE = 0: the stride is a run-time value.
+    auto stage = [&](auto nk_tag, auto stride_tag, auto check_tag, int base, int stride_rt, int slot, int slot_stride) {
+        constexpr int NK = decltype(nk_tag)::value;
+        constexpr int STRIDE = decltype(stride_tag)::value;
+        constexpr bool CHECK = decltype(check_tag)::value;
+        const int stride = STRIDE ? STRIDE : stride_rt;
+        float acc[NK];
+        bool ok[NK];
 #pragma unroll
-    for (int q = 0; q < kLen; ++q) chan[q] = Xn + (size_t)it.ch[q < m ? q : 0] * L;
-    // sum of the chosen channels at sample pos; zero outside the series (the nesting keeps the number of
-    // executed loads at the number of channels: m is the same for the whole block)
-    auto sample_at = [&](int pos) -> float {
-        if ((unsigned)pos >= (unsigned)L) return 0.0f;
-        float v = __ldg(chan[0] + pos);
-        if (m > 1) { v += __ldg(chan[1] + pos);
-        if (m > 2) { v += __ldg(chan[2] + pos);
-        if (m > 3) { v += __ldg(chan[3] + pos);
-        if (m > 4) { v += __ldg(chan[4] + pos);
-        if (m > 5) { v += __ldg(chan[5] + pos);
-        if (m > 6) { v += __ldg(chan[6] + pos);
-        if (m > 7) { v += __ldg(chan[7] + pos);
-        if (m > 8) { v += __ldg(chan[8] + pos); } } } } } } } }
-        return v;
-    };
-    const int nf = it.nf;
-    auto pool = [&](const float (&win)[kLen]) {   // one output: nine products, then Eq. 1 against every bias
-        float z = 0.0f;
-#pragma unroll
-        for (int j = 0; j < kLen; ++j) z = fmaf(w[j], win[j], z);
-#pragma unroll
-        for (int g = 0; g < kMaxFeaturesPerItem; g += 4)
-            if (g < nf) {
-#pragma unroll
-                for (int f = g; f < g + 4; ++f) cnt[f] += z > b[f] ? 1 : 0;
-            }
-    };
-    if (d < kSmallDilation) {
-        // Small dilations: adjacent threads of a column walk would sit in far-apart rows and every load would
-        // touch its own memory sector.  Instead the block stages the channel sum of a run of consecutive
-        // samples (with 4 d more on either side) in shared memory and every thread takes consecutive outputs.
-        for (int p0 = first; p0 < last; p0 += kChunk) {
-            const int lo = p0 - 4 * d, n_stage = min(kChunk, last - p0) + 8 * d;
-            __syncthreads();
-            for (int e = threadIdx.x; e < n_stage; e += kThreads) s_x[e] = sample_at(lo + e);
-            __syncthreads();
-            const int n_out = min(kChunk, last - p0);
-            for (int e = threadIdx.x; e < n_out; e += kThreads) {
-                float win[kLen];
-#pragma unroll
-                for (int j = 0; j < kLen; ++j) win[j] = s_x[e + j * d];
-                pool(win);
-            }
+        for (int k = 0; k < NK; ++k) {
+            acc[k] = 0.0f;
+            ok[k] = !CHECK || (unsigned)(base + k * stride) < (unsigned)L;
         }
-    } else {
-    constexpr int kStep = 4;   // rows fetched ahead of their use: their loads are in flight together
-    for (int u = threadIdx.x; u < n_units; u += kThreads) {
-        const int seg = u / d, r = u - seg * d;
-        const int t_a = seg * rows_per_seg, t_b = min(T, t_a + rows_per_seg);
-        // every position of the walk fits 32 bits: (T + 8) d <= L + 9 d
-        float win[kLen];
-        int pos = (t_a - 4) * d + r;                 // the sample the next window entry comes from
+        int q = 0;
+        for (; q + 2 <= m; q += 2) {
+            const float* __restrict__ x0 = Xn + s_choff[q] + base;
+            const float* __restrict__ x1 = Xn + s_choff[q + 1] + base;
+            float v0[NK], v1[NK];
 #pragma unroll
-        for (int j = 0; j < kLen - 1; ++j) { win[j + 1] = sample_at(pos); pos += d; }
-        int i = t_a * d + r;                         // the output the window is centred on next
-        for (int t0 = t_a; t0 < t_b; t0 += kStep) {
-            float nxt[kStep];
-#pragma unroll
-            for (int k = 0; k < kStep; ++k) { nxt[k] = sample_at(pos); pos += d; }
-#pragma unroll
-            for (int k = 0; k < kStep; ++k) {
-#pragma unroll
-                for (int j = 0; j < kLen - 1; ++j) win[j] = win[j + 1];
-                win[kLen - 1] = nxt[k];
-                if (t0 + k < t_b && i >= first && i < last) pool(win);
-                i += d;
+            for (int k = 0; k < NK; ++k) {
+                v0[k] = ok[k] ? load_at<STRIDE>(x0, k, stride) : 0.0f;
+                v1[k] = ok[k] ? load_at<STRIDE>(x1, k, stride) : 0.0f;
             }
+#pragma unroll
+            for (int k = 0; k < NK; ++k) acc[k] = (acc[k] + v0[k]) + v1[k];
         }
-    }
+        if (q < m) {
+            const float* __restrict__ x0 = Xn + s_choff[q] + base;
+#pragma unroll
+            for (int k = 0; k < NK; ++k)
+                if (ok[k]) acc[k] += load_at<STRIDE>(x0, k, stride);
+        }
+#pragma unroll
+        for (int k = 0; k < NK; ++k) s_x[slot + k * slot_stride] = acc[k];
+    };
+    using Strided = std::integral_constant<int, 0>;
+    using Dense = std::integral_constant<int, kThreads>;
+    using N8 = std::integral_constant<int, 8>;
+    using N4 = std::integral_constant<int, 4>;
+    using N2 = std::integral_constant<int, 2>;
+    using N1 = std::integral_constant<int, 1>;
+    using Checked = std::true_type;
+    using Inside = std::false_type;
+
+    for (int ta = 0; ta < T; ta += tile_rows) {
+        const int rows = min(tile_rows, T - ta);
+        for (int ca = 0; ca < d; ca += P) {
+            const int cols = min(P, d - ca);
+            __syncthreads();                             // the previous tile's walks are over (and s_choff is written)
+            if (whole_rows) {
+                // slots [0, count) hold positions g0 .. g0 + count: zeros before the series, the samples in
+                // rounds of 8 x 256 and of 256 without any test, one last partial round, zeros after the series
+                const int count = (rows + 8) * d, g0 = (ta - 4) * d;
+                const int z0 = min(max(-g0, 0), count), z1 = min(max(L - g0, 0), count);
+                for (int e = tid; e < z0; e += kThreads) s_x[e] = 0.0f;
+                for (int e = z1 + tid; e < count; e += kThreads) s_x[e] = 0.0f;
+                int e0 = z0;
+                for (; e0 + 8 * kThreads <= z1; e0 += 8 * kThreads) stage(N8{}, Dense{}, Inside{}, g0 + e0 + tid, 0, e0 + tid, kThreads);
+                for (; e0 + kThreads <= z1; e0 += kThreads) stage(N1{}, Dense{}, Inside{}, g0 + e0 + tid, 0, e0 + tid, kThreads);
+                if (e0 + tid < z1) stage(N1{}, Dense{}, Inside{}, g0 + e0 + tid, 0, e0 + tid, kThreads);
+            } else {
+                for (int cb = 0; cb < cols; cb += kThreads) {
+                    if (cb + tid >= cols) continue;
+                    // staged row r is row ta - 4 + r of the view: zeros above the series, rows that lie inside it
+                    // for every column of this block without any test, the rows the series ends in, zeros below
+                    const int w = min(kThreads, cols - cb), c_lo = ca + cb;
+                    const int n_rows = rows + 8;
+                    const int r_a = min(max(4 - ta, 0), n_rows);
+                    const int t_full = L >= c_lo + w ? (L - c_lo - w) / d + 1 : 0;     // rows t < t_full hold all w columns
+                    const int t_some = L > c_lo ? (L - c_lo - 1) / d + 1 : 0;          // rows t < t_some hold at least one
+                    const int r_b = min(max(t_full - (ta - 4), r_a), n_rows), r_c = min(max(t_some - (ta - 4), r_b), n_rows);
+                    const int pos0 = (ta - 4) * d + c_lo + tid, slot0 = cb + tid;
+                    for (int r = 0; r < r_a; ++r) s_x[slot0 + r * P] = 0.0f;
+                    int r = r_a;
+                    for (; r + 8 <= r_b; r += 8) stage(N8{}, Strided{}, Inside{}, pos0 + r * d, d, slot0 + r * P, P);
+                    if (r + 4 <= r_b) { stage(N4{}, Strided{}, Inside{}, pos0 + r * d, d, slot0 + r * P, P); r += 4; }
+                    if (r + 2 <= r_b) { stage(N2{}, Strided{}, Inside{}, pos0 + r * d, d, slot0 + r * P, P); r += 2; }
+                    if (r + 1 <= r_b) { stage(N1{}, Strided{}, Inside{}, pos0 + r * d, d, slot0 + r * P, P); r += 1; }
+                    for (; r < r_c; ++r) stage(N1{}, Strided{}, Checked{}, pos0 + r * d, d, slot0 + r * P, P);
+                    for (; r < n_rows; ++r) s_x[slot0 + r * P] = 0.0f;
+                }
+            }
+            __syncthreads();
+            static_assert(kMaxFeaturesPerItem == 8, "two groups of four features");
+            if (groups == 1) mini_walk_tile<1>(s_x, P, cols, rows, seg_rows, ta, ca, d, t_min, last, w, b, cnt);
+            else mini_walk_tile<2>(s_x, P, cols, rows, seg_rows, ta, ca, d, t_min, last, w, b, cnt);
+        }
     }
 #pragma unroll
     for (int f = 0; f < kMaxFeaturesPerItem; ++f) {
         const int v = __reduce_add_sync(0xffffffffu, cnt[f]);
-        if ((threadIdx.x & 31) == 0 && v) atomicAdd(&s_cnt[f], v);
+        if ((tid & 31) == 0 && v) atomicAdd(&s_cnt[f], v);
     }
     __syncthreads();
-    if (threadIdx.x < it.nf)
-        feat[(size_t)n * F + it.f0 + threadIdx.x] = (float)s_cnt[threadIdx.x] / (float)(last - first);   // Eq. 2
+    if (tid < nf) feat[(size_t)n * F + it.f0 + tid] = (float)s_cnt[tid] / (float)(last - first);   // Eq. 2
 }
 
 }  // namespace
@@ -189,8 +300,43 @@ struct rocket_mini {
 
 namespace {
 
+// Tiling of the dilated view for dilation d: the cheapest of the candidates under a simple cost model (staged
+// samples, and thread slots of the walks including the ones that idle in a partly filled round of the block).
+// Tiles either span whole rows (width = d) or 256-column multiples; runs are multiples of the window length;
+// below 32 columns only run lengths that keep the lanes of a warp on different shared-memory banks.
+void choose_tiling(int d, int L, int& width, int& seg_rows, int& segs) {
+    const int T = (L + d - 1) / d;
+    const double c_stage = 17.0, c_walk = 21.0, c_fill = 16.0;
+    double best = 1e300;
+    width = 0;
+    auto consider = [&](int w, int sr, int sg) {
+        if ((int64_t)(sg * sr + 8) * w > kTileSamples) return;
+        const int tile_rows = sr * sg;
+        double cost = 0.0;
+        for (int ta = 0; ta < T; ta += tile_rows) {
+            const int rows = std::min(tile_rows, T - ta), sgt = (rows + sr - 1) / sr;
+            for (int ca = 0; ca < d; ca += w) {
+                const int cols = std::min(w, d - ca);
+                const double rounds = std::ceil((double)cols * sgt / kThreads);
+                cost += (double)(rows + 8) * cols * c_stage + rounds * kThreads * (std::min(sr, rows) * c_walk + c_fill);
+            }
+        }
+        if (cost < best) { best = cost; width = w; seg_rows = sr; segs = sg; }
+    };
+    for (int sr = kLen; sr <= 7 * kLen; sr += kLen) {
+        if (d < 32 && sr != 3 * kLen && sr != 7 * kLen) continue;
+        const int max_segs = std::max(1, (T + sr - 1) / sr);
+        for (int sg = 1; sg <= max_segs; sg = sg < 8 ? sg + 1 : sg * 2) consider(d, sr, sg);
+        consider(d, sr, max_segs);
+        if (kTileSamples / d - 8 >= sr) consider(d, sr, std::min(max_segs, (kTileSamples / d - 8) / sr));
+        for (int w = kThreads; w < d; w += kThreads)
+            for (int sg = 1; sg <= std::min(max_segs, 4); ++sg) consider(w, sr, sg);
+    }
+}
+
 void build_items(rocket_mini& p) {
     p.items.clear();
+    std::map<int, std::array<int, 3>> tiling;           // by dilation
     for (int c = 0; c < p.n_combos; ++c)
         for (int f0 = p.feature_offset[c]; f0 < p.feature_offset[c + 1]; f0 += kMaxFeaturesPerItem) {
             MiniItem it{};
@@ -198,6 +344,13 @@ void build_items(rocket_mini& p) {
             it.f0 = f0; it.nf = std::min(kMaxFeaturesPerItem, p.feature_offset[c + 1] - f0);
             for (int k = 0; k < 3; ++k) it.tap[k] = p.taps[3 * p.kernel_index[c] + k];
             for (int q = 0; q < it.m; ++q) it.ch[q] = p.channel_idx[p.channel_offset[c] + q];
+            auto found = tiling.find(it.d);
+            if (found == tiling.end()) {
+                std::array<int, 3> t{};
+                choose_tiling(it.d, p.L, t[0], t[1], t[2]);
+                found = tiling.emplace(it.d, t).first;
+            }
+            it.width = found->second[0]; it.seg_rows = found->second[1]; it.segs = found->second[2];
             p.items.push_back(it);
         }
 }
@@ -211,6 +364,10 @@ int ensure_mini_device(const rocket_mini* p) {
         cudaError_t e = rocket::device_malloc(&p->blob, ib + bb + 256);
         if (e != cudaSuccess) { cudaGetLastError(); p->blob = nullptr; return e == cudaErrorMemoryAllocation ? ROCKET_ENOMEM : ROCKET_ECUDA; }
         if (cudaMemcpy(p->blob, p->items.data(), p->items.size() * sizeof(MiniItem), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaGetLastError(); cudaFree(p->blob); p->blob = nullptr; return ROCKET_ECUDA;
+        }
+        if (cudaFuncSetAttribute(mini_transform_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(kTileSamples * sizeof(float))) != cudaSuccess) {
             cudaGetLastError(); cudaFree(p->blob); p->blob = nullptr; return ROCKET_ECUDA;
         }
         p->d_items = static_cast<const MiniItem*>(p->blob);
@@ -236,6 +393,7 @@ extern "C" {
 
 int rocket_mini_create(uint64_t seed, int C, int L, int num_features, rocket_mini_t** out) {
     if (!out || C < 1 || L < kLen || num_features < kKernels) return ROCKET_EINVAL;
+    if ((int64_t)C * L > 0x7fffffffll) return ROCKET_EUNSUPPORTED;     // positions within an example are 32-bit
     rocket_mini* p = new (std::nothrow) rocket_mini();
     if (!p) return ROCKET_ENOMEM;
     try {
@@ -402,7 +560,7 @@ int rocket_mini_transform(const rocket_mini_t* p, const float* X_dev, int N, int
     int prev = -1;
     if (cudaGetDevice(&prev) != cudaSuccess) { cudaGetLastError(); return ROCKET_ECUDA; }
     if (prev != p->device && cudaSetDevice(p->device) != cudaSuccess) { cudaGetLastError(); return ROCKET_ECUDA; }
-    mini_transform_kernel<<<(unsigned)blocks, kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+    mini_transform_kernel<<<(unsigned)blocks, kThreads, kTileSamples * sizeof(float), static_cast<cudaStream_t>(cuda_stream)>>>(
         X_dev, C, L, p->d_items, (int)p->items.size(), p->d_bias, feat_dev, p->F);
     rocket::count_launch();
     const cudaError_t e = cudaGetLastError();
