@@ -37,8 +37,8 @@ MINI_FEATURES = 9996          # MINIROCKET's default 10,000 rounded down to a mu
 # DRAM bytes (read + write) of one launch of either fused kernel, from the committed ncu capture (profiles/),
 # per launch = one chunk of 12 examples.  The figures belong to one state of the kernel sources: they are
 # reported only while the digest of those sources still equals NCU_SOURCES_DIGEST, and as null otherwise.
-NCU_DRAM_BYTES_PER_LAUNCH = {"fast_s_forward": 56.0e6, "fast_t_forward": 313.2e6}
-NCU_SOURCES_DIGEST = "978d85d5115d532e"
+NCU_DRAM_BYTES_PER_LAUNCH = {"fast_s_forward": 56.6e6, "fast_t_forward": 311.6e6}
+NCU_SOURCES_DIGEST = "9b98ef87c1ea1846"
 KERNEL_SOURCES = ("rocket_fast_fwd.cu", "rocket_fast.h", "rocket_fast_geom.h", "rocket_plan.cpp")
 
 
@@ -431,9 +431,11 @@ def main():
         yr = torch.from_numpy((0.6 + 1.2 * rngr.random(677)).astype(np.float32)).cuda()
         rk.rocket_ridge_fit(Fr, yr, 1.0)
         torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        wr, br = rk.rocket_ridge_fit(Fr, yr, 1.0)     # returns after its work has finished
-        s_fit = time.perf_counter() - t0
+        s_fit = float("inf")
+        for _ in range(2):
+            t0 = time.perf_counter()
+            wr, br = rk.rocket_ridge_fit(Fr, yr, 1.0)     # returns after its work has finished
+            s_fit = min(s_fit, time.perf_counter() - t0)
         yhat = torch.empty((w["N"],), dtype=torch.float32, device="cuda")
         s_pred, _ = time_steps(lambda: rk.rocket_ridge_predict(feat, wr, br, out=yhat), 5, 3)
         s_pred /= 5
