@@ -336,13 +336,15 @@ int rocket_transform_soft_backward_noalloc(const rocket_params_t* p, const float
  * of the outputs of training example floor(example_draw[c] * N).
  *
  * rocket_mini_create   host only; *out owns the parameters (release with rocket_mini_destroy).  Needs C >= 1,
- *                      L >= 9, num_features >= 84.
+ *                      L >= 9, num_features >= 84 (ROCKET_EINVAL otherwise); C * L < 2^31
+ *                      (ROCKET_EUNSUPPORTED beyond: positions within an example are 32-bit).
  * rocket_mini_fit      X_host [N][C][L] fp32 on the HOST; computes every bias (a one-off over one example per
  *                      combination, on the host's cores); returns when done.
  * rocket_mini_set_biases  installs biases computed elsewhere ([n_features] floats, host).
  * rocket_mini_transform   X_dev [N][C][L] fp32 and feat_dev [N][n_features] fp32 on the device; one fused kernel
- *                      on the caller's stream (convolution outputs never reach memory); the first call binds
- *                      the handle to the current device and uploads its parameters.  ROCKET_EINVAL before
+ *                      on the caller's stream (convolution outputs never reach memory; any L, any 4-byte
+ *                      aligned X_dev); the first call binds the handle to the current device, uploads its
+ *                      parameters (one allocation) and opts the kernel into 64 KB of shared memory.  ROCKET_EINVAL before
  *                      a fit or set_biases; ROCKET_ESHAPE when C or L differ from the handle's.
  * rocket_mini_host_view   read-only views of the host arrays (taps [84][3], per combination: dilation,
  *                      kernel_index, padded, num_channels, ragged channel_idx, feature_offset [n + 1],
