@@ -53,8 +53,8 @@ def kernel_sources_digest():
 
 
 def measured_fma_peak():
-    """FP32 FMA rate of dependent register chains on this device (scalar and packed two-wide), measured with the
-    benchmark-only helper library; None when it cannot run."""
+    """FMA rate of dependent register chains on this device (scalar and packed two-wide fp32, packed fp16),
+    measured with the benchmark-only helper library; None when it cannot run."""
     import ctypes
     try:
         from paper_2301_08527_b200.build import build_bench_helper
@@ -62,7 +62,11 @@ def measured_fma_peak():
         a, b = ctypes.c_double(0.0), ctypes.c_double(0.0)
         if lib.fma_peak_measure(ctypes.byref(a), ctypes.byref(b)) != 0:
             return None
-        return {"scalar_fma_tflops": a.value, "packed_fma_tflops": b.value}
+        res = {"scalar_fma_tflops": a.value, "packed_fma_tflops": b.value}
+        h = ctypes.c_double(0.0)
+        if lib.fma_peak_measure_f16x2(ctypes.byref(h)) == 0:
+            res["packed_f16_fma_tflops"] = h.value      # fma.rn.f16x2: what a half-precision inner loop could reach
+        return res
     except Exception:
         return None
 
