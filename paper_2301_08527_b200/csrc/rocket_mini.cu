@@ -334,7 +334,8 @@ void choose_tiling(int d, int L, int& width, int& seg_rows, int& segs) {
     }
 }
 
-void build_items(rocket_mini& p) {
+// false when a dilation has no tiling that fits the shared-memory tile (cannot happen for L >= 9; checked all the same)
+bool build_items(rocket_mini& p) {
     p.items.clear();
     std::map<int, std::array<int, 3>> tiling;           // by dilation
     for (int c = 0; c < p.n_combos; ++c)
@@ -348,11 +349,13 @@ void build_items(rocket_mini& p) {
             if (found == tiling.end()) {
                 std::array<int, 3> t{};
                 choose_tiling(it.d, p.L, t[0], t[1], t[2]);
+                if (t[0] < 1 || t[1] < kLen || t[2] < 1 || (int64_t)(t[1] * t[2] + 8) * t[0] > kTileSamples) return false;
                 found = tiling.emplace(it.d, t).first;
             }
             it.width = found->second[0]; it.seg_rows = found->second[1]; it.segs = found->second[2];
             p.items.push_back(it);
         }
+    return true;
 }
 
 int ensure_mini_device(const rocket_mini* p) {
@@ -442,7 +445,10 @@ int rocket_mini_create(uint64_t seed, int C, int L, int num_features, rocket_min
         p->quantile.resize(p->F);
         for (int f = 0; f < p->F; ++f) p->quantile[f] = std::fmod((f + 1.0) * kInvGoldenRatio, 1.0);
         p->bias.assign(p->F, 0.0f);
-        build_items(*p);
+        if (!build_items(*p)) {
+            delete p;
+            return ROCKET_EUNSUPPORTED;
+        }
     } catch (const std::bad_alloc&) {
         delete p;
         return ROCKET_ENOMEM;

@@ -36,6 +36,16 @@ def test_host_fit_gives_the_oracles_biases():
     m.close()
 
 
+@pytest.mark.parametrize("L", [9, 10, 17, 63, 64, 100, 999, 4099, 50001, 200000, 1000003])
+def test_a_handle_exists_for_any_series_length(L):
+    # creation chooses, per dilation, how the kernel tiles the dilated view; every dilation of every length
+    # from the shortest (9 samples: dilation 1 only) upwards must find a tiling
+    m = rk.MiniRocket.create(3, 3, L, 84 * 12)
+    a = m.host_arrays()
+    assert a["dilation"].min() == 1 and a["dilation"].max() <= max(1, (L - 1) // 8)
+    m.close()
+
+
 def test_argument_checks():
     lib = rk.load_library()
     import ctypes
