@@ -43,6 +43,13 @@ def test_minirocket_small_full(C, L, N, F):
     _check(C, L, N, F, seed=31 + L)
 
 
+@pytest.mark.parametrize("C,L,N,F", [(2, 777, 2, 84 * 32), (5, 12001, 2, 84 * 32), (3, 30003, 1, 84 * 32), (1, 2050, 3, 84 * 64)])
+def test_minirocket_every_tile_shape(C, L, N, F):
+    # 32 dilations per kernel: tiles of whole rows and of 256-column blocks, ragged last column tiles, runs of 9
+    # to 63 rows, series lengths that are no multiple of anything
+    _check(C, L, N, F, seed=77 + L)
+
+
 def test_minirocket_univariate_random_walks():
     _check(1, 512, 16, 10000, seed=8527, series=random_walk_series)
 
