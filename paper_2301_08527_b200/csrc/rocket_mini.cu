@@ -121,28 +121,32 @@ __device__ __forceinline__ void mini_steps(const float*& p, int pitch, int left,
     }
 }
 
-// The walks over one staged tile: thread u of cols * segs takes column u % cols over run u / cols.
+// The walks over one staged tile: thread u of cols * segs takes column u % cols over run u / cols.  Outputs of
+// column c are the rows t_min <= t < t_full + (c < c_more): t d + c < last with last = t_full d + c_more.
 template <int NG>
 __device__ __forceinline__ void mini_walk_tile(const float* s_x, int P, int cols, int rows, int seg_rows, int ta, int ca,
-                                               int d, int t_min, int last, const float (&w)[kLen],
+                                               int t_min, int t_full, int c_more, const float (&w)[kLen],
                                                const float (&b)[kMaxFeaturesPerItem], int (&cnt)[kMaxFeaturesPerItem]) {
     const int segs = (rows + seg_rows - 1) / seg_rows;
+    // (run, column) of thread u, stepped without divisions: u advances by the block's threads
+    const int dq = kThreads / cols, dr = kThreads - dq * cols;
+    int seg = threadIdx.x / cols, c = threadIdx.x - seg * cols;
     for (int u = threadIdx.x; u < cols * segs; u += kThreads) {
-        const int seg = u / cols, c = u - seg * cols;
-        // rows of this run that are outputs: t >= t_min and t d + column < last
-        const int col = ca + c;
-        const int t_end = last > col ? (last - col + d - 1) / d : 0;
+        const int t_end = t_full + (ca + c < c_more ? 1 : 0);
         const int t_lo = max(ta + seg * seg_rows, t_min);
         const int t_hi = min(min(ta + rows, ta + (seg + 1) * seg_rows), t_end);
         int left = t_hi - t_lo;
-        if (left <= 0) continue;
-        // the window of output row t holds rows t - 4 .. t + 4; staged row 0 is row ta - 4
-        const float* p = s_x + (t_lo - ta) * P + c;
-        float win[kLen];
+        if (left > 0) {
+            // the window of output row t holds rows t - 4 .. t + 4; staged row 0 is row ta - 4
+            const float* p = s_x + (t_lo - ta) * P + c;
+            float win[kLen];
 #pragma unroll
-        for (int j = 0; j < kLen - 1; ++j) { win[j] = *p; p += P; }
-        for (; left >= kLen; left -= kLen) mini_steps<0, false, NG>(p, P, left, win, w, b, cnt);
-        mini_steps<0, true, NG>(p, P, left, win, w, b, cnt);
+            for (int j = 0; j < kLen - 1; ++j) { win[j] = *p; p += P; }
+            for (; left >= kLen; left -= kLen) mini_steps<0, false, NG>(p, P, left, win, w, b, cnt);
+            if (left > 0) mini_steps<0, true, NG>(p, P, left, win, w, b, cnt);
+        }
+        seg += dq; c += dr;
+        if (c >= cols) { c -= cols; ++seg; }
     }
 }
 
@@ -180,6 +184,7 @@ mini_transform_kernel(const float* __restrict__ X, int C, int L, const MiniItem*
     const int tile_rows = seg_rows * it.segs;
     const bool whole_rows = P == d;                      // a tile spans whole rows: its samples are one contiguous run
     const int t_min = it.padded ? 0 : 4;                 // rows below hold no output of an unpadded combination
+    const int t_full = last / d, c_more = last - t_full * d;   // column c has outputs in rows t < t_full + (c < c_more)
     const int groups = (nf + 3) / 4;
 
     // NK staged samples per thread at a time: position base + k * stride goes to slot + k * slot_stride.  The
@@ -268,8 +273,8 @@ mini_transform_kernel(const float* __restrict__ X, int C, int L, const MiniItem*
             }
             __syncthreads();
             static_assert(kMaxFeaturesPerItem == 8, "two groups of four features");
-            if (groups == 1) mini_walk_tile<1>(s_x, P, cols, rows, seg_rows, ta, ca, d, t_min, last, w, b, cnt);
-            else mini_walk_tile<2>(s_x, P, cols, rows, seg_rows, ta, ca, d, t_min, last, w, b, cnt);
+            if (groups == 1) mini_walk_tile<1>(s_x, P, cols, rows, seg_rows, ta, ca, t_min, t_full, c_more, w, b, cnt);
+            else mini_walk_tile<2>(s_x, P, cols, rows, seg_rows, ta, ca, t_min, t_full, c_more, w, b, cnt);
         }
     }
 #pragma unroll
