@@ -326,7 +326,8 @@ int rocket_transform_soft_backward_noalloc(const rocket_params_t* p, const float
  * What the paper leaves open is fixed as follows.  Kernels: the 84 ways to give three of nine taps the weight
  * 2 and the other six -1.  num_features is rounded down to a multiple of 84 (10,000 -> 9,996); every kernel
  * owns the same number of features, spread over the distinct values of floor(2^x), x equally spaced on
- * [0, log2((L - 1) / 8)] (at most 32 of them).  Combination c = dilation_index * 84 + kernel_index owns the
+ * [0, log2((L - 1) / 8)] (at most 32 of them; computed as floor(exp2(x) * (1 + 2^-40)) in double precision, so
+ * that a power that is an integer - the largest is (L - 1) / 8 itself - is not lost to a rounding error).  Combination c = dilation_index * 84 + kernel_index owns the
  * features feature_offset[c] .. feature_offset[c + 1] - 1, has padding 4 d (outputs 0 .. L - 1) when
  * dilation_index + kernel_index is even and none otherwise (outputs 4 d .. L - 4 d - 1), and a random subset of
  * floor(2^U(0, log2(min(C, 9) + 1))) channels whose samples are summed before the convolution (the same

@@ -416,7 +416,8 @@ int rocket_mini_create(uint64_t seed, int C, int L, int num_features, rocket_min
         std::vector<int64_t> count;
         for (int k = 0; k < n; ++k) {
             const double x = n > 1 ? k * E / (n - 1) : 0.0;
-            const int64_t d = (int64_t)std::floor(std::exp2(x));
+            // a power that is an integer (the last one is (L - 1) / 8) must not fall below it by exp2's rounding
+            const int64_t d = (int64_t)std::floor(std::exp2(x) * (1.0 + 0x1.0p-40));
             if (!dil.empty() && dil.back() == d) ++count.back();
             else { dil.push_back(d); count.push_back(1); }
         }

@@ -10,7 +10,9 @@ oracle and to the library.
   kernels       the 84 ways to give three of nine taps the weight 2 and the other six the weight -1 (every
                 kernel sums to zero), in lexicographic order of the three positions
   features      F is rounded down to a multiple of 84; every kernel owns F / 84 features, spread over dilations
-  dilations     with n = min(F / 84, 32): floor(2^(k E / (n - 1))), k = 0..n-1, E = log2((L - 1) / 8); equal
+  dilations     with n = min(F / 84, 32): floor(2^(k E / (n - 1)) (1 + 2^-40)), k = 0..n-1, E = log2((L - 1) / 8)
+                (the factor keeps a power that is an integer - the last one is (L - 1) / 8 - from falling below it
+                by a rounding error of exp2); equal
                 values merge, a merged value keeps the sum of their shares of the F / 84 features (shares are
                 floored, what is left over goes one by one to the smallest dilations)
   combination   c = dilation_index * 84 + kernel_index owns n_features[c] consecutive features
@@ -81,7 +83,7 @@ def dilations_and_shares(L, F):
     n = min(fpk, 32)
     E = np.log2((L - 1.0) / 8.0)
     exps = np.array([k * E / (n - 1) for k in range(n)]) if n > 1 else np.zeros(1)
-    raw = np.floor(np.exp2(exps)).astype(np.int64)
+    raw = np.floor(np.exp2(exps) * (1.0 + 2.0 ** -40)).astype(np.int64)   # an integer value counts as itself, whatever exp2 rounds to
     dil, counts = np.unique(raw, return_counts=True)
     share = np.floor(counts * (fpk / n)).astype(np.int64)
     left = fpk - int(share.sum())

@@ -38,7 +38,8 @@ def _check(C, L, N, F, seed, series=ar1_spike_series, examples=None):
     return P.check_hard_ppv(feat[sel], band)
 
 
-@pytest.mark.parametrize("C,L,N,F", [(3, 700, 3, 84 * 12), (1, 64, 4, 84 * 40), (20, 5000, 4, 10000), (2, 9, 3, 84), (7, 4099, 2, 84 * 20)])
+@pytest.mark.parametrize("C,L,N,F", [(3, 700, 3, 84 * 12), (1, 64, 4, 84 * 40), (20, 5000, 4, 10000), (2, 9, 3, 84), (7, 4099, 2, 84 * 20),
+                                     (5, 49, 1, 168)])
 def test_minirocket_small_full(C, L, N, F):
     _check(C, L, N, F, seed=31 + L)
 

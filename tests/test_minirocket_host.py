@@ -8,7 +8,8 @@ import paper_2301_08527_b200 as rk
 from rocket_inputs import ar1_spike_series, generate_minirocket
 
 
-@pytest.mark.parametrize("C,L,F", [(1, 64, 500), (20, 5000, 10000), (5, 50000, 10000), (9, 300, 84)])
+@pytest.mark.parametrize("C,L,F", [(1, 64, 500), (20, 5000, 10000), (5, 50000, 10000), (9, 300, 84), (5, 49, 168), (3, 57, 840),
+                                   (2, 4097, 2688), (4, 1001, 1680), (2, 9, 84), (1, 25, 252)])
 def test_library_parameters_equal_the_reference_generator(C, L, F):
     ref = generate_minirocket(8527, C, L, F)
     m = rk.MiniRocket.create(8527, C, L, F)
