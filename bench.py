@@ -71,6 +71,43 @@ def measured_fma_peak():
         return None
 
 
+def run_gemm_probe():
+    """The transform of one dilation as a GEMM: Z[kernels][positions] = W'[kernels][K] X_d[K][positions] with the
+    weights of every kernel laid out on a common grid of 11 centred taps x 24 channel slots (K = 264), of which a
+    kernel fills 31.6 on average.  Times the library GEMM (fp32, tf32, bf16 inputs) for bucket sizes M and reports
+    dense and useful TFLOP/s; an upper bound for a tensor-core form, which would also have to build X_d (every
+    channel row 11 times, shifted) and pool the outputs."""
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    K, N = 264, 600000                       # 12 examples x 50,000 positions
+    useful = 31.6 / K
+    rows = []
+    for M in (64, 128, 256, 768):
+        for name, dtype, tf32 in (("fp32", torch.float32, False), ("tf32", torch.float32, True), ("bf16", torch.bfloat16, False)):
+            torch.backends.cuda.matmul.allow_tf32 = tf32
+            A = torch.randn(M, K, device="cuda", dtype=dtype)
+            B = torch.randn(K, N, device="cuda", dtype=dtype)
+            C = torch.empty(M, N, device="cuda", dtype=dtype)
+            for _ in range(3):
+                torch.matmul(A, B, out=C)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(10):
+                torch.matmul(A, B, out=C)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / 10
+            dense = 2.0 * M * N * K / ms / 1e9
+            rows.append({"M": M, "inputs": name, "ms": ms, "dense_tflops": dense, "useful_tflops": dense * useful,
+                         "useful_tflops_three_products": dense * useful / 3})
+            del A, B, C
+    torch.backends.cuda.matmul.allow_tf32 = False
+    print(json.dumps({"probe": "library GEMM, zero-padded dense-channel formulation", "K": K, "N": N,
+                      "useful_share_of_K": useful, "rows": rows}))
+
+
 def fp32_peak_tflops(sm_count, sm_mhz):
     """FP32 FMA peak: SMs x 128 lanes x 2 flop x clock."""
     return sm_count * 128 * 2 * sm_mhz * 1e6 / 1e12
@@ -223,7 +260,14 @@ def main():
     ap.add_argument("--profile-pass", choices=["soft", "backward", "minirocket"], default=None,
                     help="profiling case: run only that pass (config 3's soft forward or backward, or the MINIROCKET "
                          "transform with 9,996 features) on 12 examples, three times, and exit")
+    ap.add_argument("--gemm-probe", action="store_true",
+                    help="measure what a library GEMM makes of the zero-padded dense-channel formulation of the transform "
+                         "(a reference measurement for the design notes: the transform itself never calls a GEMM) and exit")
     args = ap.parse_args()
+
+    if args.gemm_probe:
+        run_gemm_probe()
+        return
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
