@@ -15,17 +15,18 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "rocket_oracle.c")
 _SRC_MINI = os.path.join(_HERE, "minirocket_oracle.c")
+_SRC_F16 = os.path.join(_HERE, "rocket_f16_oracle.c")
 _LIB = os.path.join(_HERE, "_build", "librocket_oracle.so")
 _lib = None
 
 
 def build(force=False):
     """Compile the oracle with gcc (-O2, OpenMP).  Returns the path of the shared object."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_MINI)):
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_MINI), os.path.getmtime(_SRC_F16)):
         os.makedirs(os.path.dirname(_LIB), exist_ok=True)
         tmp = _LIB + ".%d.tmp" % os.getpid()
         subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
-                               "-ffp-contract=off", "-o", tmp, _SRC, _SRC_MINI, "-lm"])
+                               "-ffp-contract=off", "-o", tmp, _SRC, _SRC_MINI, _SRC_F16, "-lm"])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -197,6 +198,55 @@ def backward(p, X, g, argmax, lam=1.0, shift=3.0, examples=None, kernels=None):
                                _ptr(ks), ctypes.c_double(lam), ctypes.c_double(shift), _ptr(g), _ptr(argmax),
                                _ptr(dW), _ptr(db))
     return dW, db
+
+
+# ---- half-precision transform (oracle/rocket_f16_oracle.c) ---------------------------------------------------
+
+def round_f16(a):
+    """The binary16 numbers nearest to a (ties to even), as float32."""
+    with np.errstate(over="raise"):
+        return np.asarray(a, np.float32).astype(np.float16).astype(np.float32)
+
+
+def forward_f16_pairs(p, X, pair_n, pair_k, return_z=False):
+    """Half-precision hard transform for explicit (example, kernel) pairs: samples, weights and biases are rounded
+    to binary16 here, every multiply-add of the convolution rounds once to binary16 (bias first, then the channels
+    in the kernel's order, taps 0 .. len - 1).  Returns a namespace of 1-D arrays: count (int64), ppv, max
+    (float64), argmax (int32), out_len; with return_z also z (the outputs of the first pair)."""
+    import copy
+    lib = _load()
+    X16 = round_f16(_check_x(p, X))
+    p16 = copy.copy(p)
+    p16.weights = round_f16(p.weights)
+    p16.bias = round_f16(p.bias)
+    pn = np.ascontiguousarray(pair_n, np.int32)
+    pk = np.ascontiguousarray(pair_k, np.int32)
+    if pn.shape != pk.shape or pn.ndim != 1:
+        raise ValueError("pair_n and pair_k must be 1-D and of equal length")
+    P = len(pn)
+    out = SimpleNamespace(count=np.empty(P, np.int64), ppv=np.empty(P), max=np.empty(P), argmax=np.empty(P, np.int32))
+    z = np.empty(int(p.out_len[pk[0]]) if (return_z and P) else 0)
+    s, keep = _cparams(p16)
+    lib.rocket_oracle_f16_forward_pairs.restype = ctypes.c_int
+    rc = lib.rocket_oracle_f16_forward_pairs(ctypes.byref(s), _ptr(X16), ctypes.c_int64(P), _ptr(pn), _ptr(pk), _ptr(out.count),
+                                             _ptr(out.ppv), _ptr(out.max), _ptr(out.argmax), _ptr(z) if return_z and P else None)
+    if rc != 0:
+        raise FloatingPointError("an input is no binary16 number or an intermediate result overflows binary16")
+    out.out_len = p.out_len[pk]
+    if return_z:
+        out.z = z
+    return out
+
+
+def forward_f16(p, X):
+    """forward_f16_pairs for every (example, kernel): each field reshaped to [N, K]."""
+    N = np.asarray(X).shape[0]
+    pn = np.repeat(np.arange(N, dtype=np.int32), p.K)
+    pk = np.tile(np.arange(p.K, dtype=np.int32), N)
+    out = forward_f16_pairs(p, X, pn, pk)
+    for name, v in vars(out).items():
+        setattr(out, name, v.reshape(N, p.K))
+    return out
 
 
 # ---- MINIROCKET (oracle/minirocket_oracle.c) ---------------------------------------------------------------
