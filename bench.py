@@ -488,6 +488,9 @@ def main():
         s_pred, _ = time_steps(lambda: rk.rocket_ridge_predict(feat, wr, br, out=yhat), 5, 3)
         s_pred /= 5
         del Fr
+        # the hard transform in half precision (Section 5: FP16 compute), device-resident input
+        s_f16, _ = time_steps(lambda: rk.rocket_transform_f16(params, X, out=feat), psteps, 3)
+        s_f16 = max_over(s_f16) / psteps
         # MINIROCKET on the same batch (Section 2; Section 6, last sentence): host fit, then the fused transform
         mr = rk.MiniRocket.create(PARAM_SEED, w["C"], w["L"], MINI_FEATURES)
         t0 = time.perf_counter()
@@ -499,6 +502,9 @@ def main():
         mr.close()
         del mfeat
         passes = {
+            "hard_f16": {"shape": "N=%d x C=%d x L=%d, K=%d, binary16 arithmetic" % (w["N"], w["C"], w["L"], w["K"]),
+                         "examples_per_s": world * w["N"] / s_f16, "ms": 1e3 * s_f16,
+                         "conv_tflops": flops_ex * w["N"] / s_f16 / 1e12},
             "minirocket": {"shape": "N=%d x C=%d x L=%d, %d features" % (w["N"], w["C"], w["L"], MINI_FEATURES),
                            "examples_per_s": world * w["N"] / s_mini, "ms": 1e3 * s_mini, "host_fit_s": s_mfit},
             "ridge": {"fit_ms": 1e3 * s_fit, "fit_shape": "677 examples x %d features, alpha=1" % (2 * w["K"]),

@@ -153,6 +153,20 @@ int rocket_transform(const rocket_params_t* p, const float* X_dev, int N, int C,
                      void* cuda_stream);
 
 /*
+ * Hard transform in half precision (Section 5 of the paper names FP16 compute as a further speed-up).  Same
+ * arguments and layout as rocket_transform.  What it computes: samples, weights and biases rounded to binary16
+ * (nearest, ties to even); every conv output starts at the bias and takes one fused multiply-add per tap -
+ * channels in the order of the kernel's channel list, taps 0 .. len - 1 - each rounded once to binary16; PPV
+ * (strict) and max of those outputs, the max returned exactly, PPV as count / L_out in fp32.  Errors against the
+ * FP32 transform are of the order of 1e-3 (PPV) and 1e-3 of the max; on this hardware the gain in speed is small
+ * (packed half-precision and packed FP32 multiply-adds issue at the same rate).  Served by the fused kernels
+ * only: ROCKET_EUNSUPPORTED when the handle has a kernel they do not take (a length other than 7, 9, 11, more
+ * than 20 channels); ROCKET_EINVAL for a base that is not 4-byte aligned; samples beyond +-65504 overflow.
+ */
+int rocket_transform_f16(const rocket_params_t* p, const float* X_dev, int N, int C, int L, float* feat_dev,
+                         void* cuda_stream);
+
+/*
  * Soft transform: softPPV (Eq. 3-4) with softness lambda and shift (Eq. 3 as printed: shift =
  * +3; the accompanying prose describes shift = -3; both are valid arguments), and max.
  *   argmax_dev [N][K] int32, device, written when not NULL: the lowest output index attaining

@@ -7,11 +7,11 @@ can be checked), but every compute call needs a CUDA device and the compiled lib
 from .binding import (MiniRocket, PASS_BACKWARD, PASS_HARD, PASS_SOFT, PASS_U8_INPUT, RocketError, RocketParams, device_alloc_count,
                       kernel_launch_count, library_path, load_library,
                       rocket_ridge_fit, rocket_ridge_predict,
-                      rocket_transform, rocket_transform_soft, rocket_transform_soft_backward, rocket_transform_soft_u8,
+                      rocket_transform, rocket_transform_f16, rocket_transform_soft, rocket_transform_soft_backward, rocket_transform_soft_u8,
                       rocket_transform_u8)
 
 __all__ = ["MiniRocket", "PASS_BACKWARD", "PASS_HARD", "PASS_SOFT", "PASS_U8_INPUT", "RocketError", "RocketParams",
            "device_alloc_count", "kernel_launch_count", "library_path", "load_library",
            "rocket_ridge_fit", "rocket_ridge_predict",
-           "rocket_transform", "rocket_transform_soft", "rocket_transform_soft_backward", "rocket_transform_soft_u8",
+           "rocket_transform", "rocket_transform_f16", "rocket_transform_soft", "rocket_transform_soft_backward", "rocket_transform_soft_u8",
            "rocket_transform_u8"]

@@ -53,6 +53,8 @@ SIGNATURES = {
     "rocket_mini_destroy": (None, [ctypes.c_void_p]),
     "rocket_transform": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                         ctypes.c_void_p, ctypes.c_void_p]),
+    "rocket_transform_f16": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                            ctypes.c_void_p, ctypes.c_void_p]),
     "rocket_transform_soft": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                                              ctypes.c_int, ctypes.c_float, ctypes.c_float, ctypes.c_void_p,
                                              ctypes.c_void_p, ctypes.c_void_p]),
@@ -263,6 +265,16 @@ def rocket_transform(params, X, out=None):
     feat = out if out is not None else torch.empty((N, 2 * params.K), dtype=torch.float32, device=X.device)
     _check(load_library().rocket_transform(params.handle, _dev_ptr(X, torch.float32, "X"), N, C, L,
                                            _dev_ptr(feat, torch.float32, "out"), _stream()), "rocket_transform")
+    return feat
+
+
+def rocket_transform_f16(params, X, out=None):
+    """Hard PPV + max in half precision (binary16 samples, weights and biases; one rounding per multiply-add)."""
+    import torch
+    N, C, L = _check_x(params, X)
+    feat = out if out is not None else torch.empty((N, 2 * params.K), dtype=torch.float32, device=X.device)
+    _check(load_library().rocket_transform_f16(params.handle, _dev_ptr(X, torch.float32, "X"), N, C, L,
+                                               _dev_ptr(feat, torch.float32, "out"), _stream()), "rocket_transform_f16")
     return feat
 
 

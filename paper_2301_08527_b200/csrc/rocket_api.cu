@@ -395,6 +395,22 @@ int rocket_transform(const rocket_params_t* p, const float* X_dev, int N, int C,
     return cuda_status(launch_generic_forward(p->dp, X_dev, N, false, 0.0f, 0.0f, feat_dev, nullptr, stream));
 }
 
+// Half-precision form of the hard transform (Section 5, "FP16 compute"): fused kernels only.
+int rocket_transform_f16(const rocket_params_t* p, const float* X_dev, int N, int C, int L, float* feat_dev,
+                         void* cuda_stream) {
+    int st = check_call(p, X_dev, N, C, L);
+    if (st != ROCKET_OK) return st;
+    if (N == 0) return ROCKET_OK;
+    if (!feat_dev) return ROCKET_EINVAL;
+    if ((st = ensure_device(p)) != ROCKET_OK) return st;
+    if (!p->fast->host.enabled || p->fast->dev.n_generic != 0) return ROCKET_EUNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(X_dev) & 3u) != 0) return ROCKET_EINVAL;
+    DeviceGuard g(p->device);
+    if (!g.ok) return ROCKET_ECUDA;
+    return cuda_status(fast::launch_fast_forward(*p->fast, p->dp, X_dev, N, feat_dev, static_cast<cudaStream_t>(cuda_stream),
+                                                 false, 0.0f, 0.0f, nullptr, nullptr, nullptr, true));
+}
+
 int rocket_transform_soft(const rocket_params_t* p, const float* X_dev, int N, int C, int L, float lambda,
                           float shift, float* feat_dev, int32_t* argmax_dev, void* cuda_stream) {
     int st = check_call(p, X_dev, N, C, L);

@@ -240,10 +240,12 @@ cudaError_t launch_fast_backward(FastState& fs, const DeviceParams& dp, int64_t 
 // Forward through the fast path: init, pad copy, S kernel, T kernel, finalise.  soft = false:
 // PPV + max; soft = true: softPPV + max (+ argmax when argmax != nullptr).
 // With X_u8 (raw 8-bit intensities [N][C][L], 4-byte aligned) the samples are normalised per channel
-// with *norm while the zero-margined copies are written, and X is not read.
+// with *norm while the zero-margined copies are written, and X is not read.  half (hard transform only): samples,
+// weights and biases are rounded to binary16 and every multiply-add of the convolution rounds once to binary16.
 cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const float* X, int N, float* feat,
                                 cudaStream_t stream, bool soft = false, float lambda = 0.0f, float shift = 0.0f,
-                                int32_t* argmax = nullptr, const uint8_t* X_u8 = nullptr, const NormArgs* norm = nullptr);
+                                int32_t* argmax = nullptr, const uint8_t* X_u8 = nullptr, const NormArgs* norm = nullptr,
+                                bool half = false);
 
 }  // namespace fast
 }  // namespace rocket

@@ -102,6 +102,68 @@ __device__ __forceinline__ void conv_channel(const float* __restrict__ st, const
     }
 }
 
+// ---- half precision (mode 3): binary16 samples, weights and bias, every multiply-add rounded once to binary16 ----
+typedef uint32_t h2;   // two binary16 numbers: the thread's column pair
+__device__ __forceinline__ h2 to_h2(float lo, float hi) {   // round to nearest even, both halves
+    h2 r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ void hfma2(h2& acc, h2 a, h2 b) {
+    asm("fma.rn.f16x2 %0, %1, %2, %0;" : "+r"(acc) : "r"(a), "r"(b));
+}
+// The pair as two floats (exact); a negative zero (a tiny negative result rounded to zero) becomes +0, so that
+// the sign bit means "below zero" as it does for the FP32 accumulators.
+__device__ __forceinline__ u64 h2_to_pair(h2 v) {
+    asm("add.rn.f16x2 %0, %0, %1;" : "+r"(v) : "r"(0u));
+    unsigned short lo, hi;
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(v));
+    float a, b;
+    asm("cvt.f32.f16 %0, %1;" : "=f"(a) : "h"(lo));
+    asm("cvt.f32.f16 %0, %1;" : "=f"(b) : "h"(hi));
+    return pack2(a, b);
+}
+// conv_channel in half precision: the FP32 samples of the staged tile and the FP32 weights of the record are
+// rounded to binary16 on the way (the same value every time it is used), the accumulators hold 0 - z as binary16.
+template <int ELL, int STEP, bool WIN, int R>
+__device__ __forceinline__ void conv_channel_h(const float* __restrict__ st, const int (&off)[4],
+                                               const float* __restrict__ w2, h2 (&acc)[R], int gl = 0, int gh = 0) {
+    h2 wp[ELL];
+#pragma unroll
+    for (int j = 0; j < ELL; ++j) {
+        const float2 v = *reinterpret_cast<const float2*>(w2 + 2 * j);
+        wp[j] = to_h2(v.x, v.y);
+    }
+#pragma unroll
+    for (int g = 0; g < (R + ELL - 1 + 3) / 4; ++g) {
+        if (!WIN || (g >= gl && g < gh)) {
+#pragma unroll
+            for (int s = 4 * g; s < 4 * g + 4 && s < R + ELL - 1; ++s) {
+                const float2 xf = *reinterpret_cast<const float2*>(st + off[s & 3] + (s >> 2) * STEP);
+                const h2 x = to_h2(xf.x, xf.y);
+#pragma unroll
+                for (int j = 0; j < ELL; ++j) {
+                    const int o = s - j;
+                    if (o >= 0 && o < R) hfma2(acc[o], wp[j], x);
+                }
+            }
+        }
+    }
+}
+// The accumulators of a tile in half precision start at 0 - bias (rounded to binary16; +0 when it rounds to zero).
+template <int R>
+__device__ __forceinline__ void init_acc_h(h2 (&acc)[R], float negb) {
+    h2 v = to_h2(negb, negb);
+    if ((v & 0x7fff7fffu) == 0u) v = 0u;
+#pragma unroll
+    for (int o = 0; o < R; ++o) acc[o] = v;
+}
+template <int R>
+__device__ __forceinline__ void widen_acc(const h2 (&acch)[R], u64 (&acc)[R]) {
+#pragma unroll
+    for (int o = 0; o < R; ++o) acc[o] = h2_to_pair(acch[o]);
+}
+
 // Adds the PPV count of the thread's 2 x 16 outputs to cnt and folds their min(-z) into mn.  Outputs outside the kernel's range
 // never need a test here: their accumulators start at +inf and stay there (sign bit clear,
 // neutral for the min).
@@ -406,7 +468,16 @@ __device__ __forceinline__ void s_kernel_tile(const float* planes, const KRec* r
         conv_channel<ELL, 4 * kWarpCols, false, false, kRS>(planes + rec->ch[q] * kSPlaneFloats, off, rec->w2[q], acc);
 }
 
-template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft
+// The same in half precision (mode 3).
+template <int ELL>
+__device__ __forceinline__ void s_kernel_tile_h(const float* planes, const KRec* rec, int lane, h2 (&acc)[kRS]) {
+    const int m = rec->m;
+    const int off[4] = {2 * lane, kWarpCols + 2 * lane, 2 * kWarpCols + 2 * lane, 3 * kWarpCols + 2 * lane};
+    for (int q = 0; q < m; ++q)
+        conv_channel_h<ELL, 4 * kWarpCols, false, kRS>(planes + rec->ch[q] * kSPlaneFloats, off, rec->w2[q], acc);
+}
+
+template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft, 3 = hard in half precision
 __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
     float* planes = reinterpret_cast<float*>(smem_raw);                               // [C][kRowsMax][64]
     KRec* recs = reinterpret_cast<KRec*>(planes + a.C * kSPlaneFloats);                // [warps][2]
@@ -496,10 +567,19 @@ __global__ void __launch_bounds__(kSThreads, 1) fast_s_forward(FwdArgs a) {
             // hard mode: the pooling masks the outputs that do not exist, so the accumulators always start inside
             // the first channel's pass; the other modes start them at 0 - bias, or +inf where there is no output
             constexpr bool kFold = MODE == 0;
-            if (!kFold) init_acc(acc, rec->negb, interior, lo0, hi0, lo1, hi1);
-            if (len == 7) s_kernel_tile<7, kFold>(planes, rec, lane, acc);
-            else if (len == 9) s_kernel_tile<9, kFold>(planes, rec, lane, acc);
-            else s_kernel_tile<11, kFold>(planes, rec, lane, acc);
+            if constexpr (MODE == 3) {
+                h2 acch[kRS];
+                init_acc_h(acch, rec->negb);
+                if (len == 7) s_kernel_tile_h<7>(planes, rec, lane, acch);
+                else if (len == 9) s_kernel_tile_h<9>(planes, rec, lane, acch);
+                else s_kernel_tile_h<11>(planes, rec, lane, acch);
+                widen_acc(acch, acc);
+            } else {
+                if (!kFold) init_acc(acc, rec->negb, interior, lo0, hi0, lo1, hi1);
+                if (len == 7) s_kernel_tile<7, kFold>(planes, rec, lane, acc);
+                else if (len == 9) s_kernel_tile<9, kFold>(planes, rec, lane, acc);
+                else s_kernel_tile<11, kFold>(planes, rec, lane, acc);
+            }
             if (MODE == 2) {
                 const int64_t pair = (int64_t)n * a.K + korig;
                 const float gP = __ldg(a.dfeat + 2 * pair), gM = __ldg(a.dfeat + 2 * pair + 1);
@@ -660,7 +740,32 @@ __device__ __forceinline__ bool t_dispatch(int len, const float* stages, const K
     return t_channels<11, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
 }
 
-template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft
+// The channels of one tile in half precision (mode 3).
+template <int ELL, int STEP, bool WIN>
+__device__ __forceinline__ bool t_channels_h(const float* stages, const KRec* rec, const int (&off)[4], uint32_t full0,
+                                             uint32_t empty0, uint32_t& st, int lane, bool active, h2 (&acc)[kR], int gl,
+                                             int gh) {
+    const int m = rec->m;
+    for (int q = 0; q < m; ++q) {
+        const uint32_t slot = st % kTStages;
+        if (q > 0 && !mbar_wait(full0 + 8u * slot, (st / kTStages) & 1u)) return false;
+        if (active) conv_channel_h<ELL, STEP, WIN, kR>(stages + slot * kTStageFloats, off, rec->w2[q], acc, gl, gh);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8u * slot);
+        ++st;
+    }
+    return true;
+}
+template <int STEP, bool WIN>
+__device__ __forceinline__ bool t_dispatch_h(int len, const float* stages, const KRec* rec, const int (&off)[4],
+                                             uint32_t full0, uint32_t empty0, uint32_t& st, int lane, bool active,
+                                             h2 (&acc)[kR], int gl, int gh) {
+    if (len == 7) return t_channels_h<7, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
+    if (len == 9) return t_channels_h<9, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
+    return t_channels_h<11, STEP, WIN>(stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
+}
+
+template <int MODE>  // 0 = hard, 1 = soft, 2 = backward of soft, 3 = hard in half precision
 __global__ void __launch_bounds__(kTBlockThreads, kTBlocksPerSM) fast_t_forward(FwdArgs a) {
     __shared__ __align__(16) TShared shs[kTGroups];
     // the block's groups work independently of one another: each has its part of the shared memory
@@ -834,11 +939,21 @@ __global__ void __launch_bounds__(kTBlockThreads, kTBlocksPerSM) fast_t_forward(
             // The other modes start at +inf where there is no output.  (Starting the accumulators inside the first
             // channel's pass, as the small-dilation kernel does, doubles the inner-loop instances here: measured
             // slower, the kernel then waits for instructions.)
-            if (active) init_acc(acc, rec->negb, interior || MODE == 0, lo0, hi0, lo1, hi1);
-            if (wide) ok = t_dispatch<kTWideCols, true>(len, stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
-            else if (cg == 1) ok = t_dispatch<kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
-            else if (cg == 2) ok = t_dispatch<2 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
-            else ok = t_dispatch<4 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
+            if constexpr (MODE == 3) {
+                h2 acch[kR];
+                init_acc_h(acch, rec->negb);
+                if (wide) ok = t_dispatch_h<kTWideCols, true>(len, stages, rec, off, full0, empty0, st, lane, active, acch, gl, gh);
+                else if (cg == 1) ok = t_dispatch_h<kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acch, 0, 0);
+                else if (cg == 2) ok = t_dispatch_h<2 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acch, 0, 0);
+                else ok = t_dispatch_h<4 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acch, 0, 0);
+                widen_acc(acch, acc);
+            } else {
+                if (active) init_acc(acc, rec->negb, interior || MODE == 0, lo0, hi0, lo1, hi1);
+                if (wide) ok = t_dispatch<kTWideCols, true>(len, stages, rec, off, full0, empty0, st, lane, active, acc, gl, gh);
+                else if (cg == 1) ok = t_dispatch<kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
+                else if (cg == 2) ok = t_dispatch<2 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
+                else ok = t_dispatch<4 * kWarpCols, false>(len, stages, rec, off, full0, empty0, st, lane, active, acc, 0, 0);
+            }
             if (!ok) break;
             const int64_t pair = (int64_t)n * a.K + korig;
             if (MODE == 2) {
@@ -883,7 +998,7 @@ __global__ void __launch_bounds__(kTBlockThreads, kTBlocksPerSM) fast_t_forward(
         }
         // what the warp still carries is published even when a wait gave up: counts and maxima are only
         // ever combined with commutative atomics, and the error flag marks the result as incomplete
-        if (MODE == 0 && cur_pair >= 0) publish(a.feat_i, cur_pair, cnt, mn, lane);
+        if ((MODE == 0 || MODE == 3) && cur_pair >= 0) publish(a.feat_i, cur_pair, cnt, mn, lane);
         if (!ok) {
             *abort_flag = 1;
             if (lane == 0) atomicExch(a.plan.error_flag, 1);
@@ -1032,6 +1147,10 @@ cudaError_t set_kernel_attributes(int dev) {
         e = cudaFuncSetAttribute(fast_s_forward<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s_smem_bytes(kSMaxChannels));
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(fast_t_forward<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t_bytes);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(fast_s_forward<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s_smem_bytes(kSMaxChannels));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(fast_t_forward<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t_bytes);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -1248,7 +1367,8 @@ cudaError_t reserve_fast_state(FastState& fs, const DeviceParams& dp, int max_N,
 
 cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const float* X, int N, float* feat,
                                 cudaStream_t stream, bool soft, float lambda, float shift, int32_t* argmax,
-                                const uint8_t* X_u8, const NormArgs* norm) {
+                                const uint8_t* X_u8, const NormArgs* norm, bool half) {
+    if (half && soft) return cudaErrorInvalidValue;
     std::lock_guard<std::mutex> lk(fs.mu);
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -1315,6 +1435,7 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
             const unsigned long long total = (unsigned long long)nc * pd.n_sitems;
             const unsigned grid = (unsigned)std::min<unsigned long long>(total, (unsigned long long)sms);
             if (soft) fast_s_forward<1><<<grid, kSThreads, s_bytes, stream>>>(a);
+            else if (half) fast_s_forward<3><<<grid, kSThreads, s_bytes, stream>>>(a);
             else fast_s_forward<0><<<grid, kSThreads, s_bytes, stream>>>(a);
             count_launch();
         }
@@ -1322,6 +1443,7 @@ cudaError_t launch_fast_forward(FastState& fs, const DeviceParams& dp, const flo
         if (pd.n_titems > 0) {
             const unsigned grid = t_grid(nc, pd.n_titems, sms);
             if (soft) fast_t_forward<1><<<grid, kTBlockThreads, t_bytes, stream>>>(a);
+            else if (half) fast_t_forward<3><<<grid, kTBlockThreads, t_bytes, stream>>>(a);
             else fast_t_forward<0><<<grid, kTBlockThreads, t_bytes, stream>>>(a);
             count_launch();
         }
