@@ -257,9 +257,10 @@ def main():
                     "calls each) on rank 0 instead of its time-boxed default (12 points, one timed call each)")
     ap.add_argument("--skip-sweep", action="store_true", help="skip the throughput sweep")
     ap.add_argument("--small", action="store_true", help="profiling case: N=12 examples, one launch of either fused kernel")
-    ap.add_argument("--profile-pass", choices=["soft", "backward", "minirocket"], default=None,
-                    help="profiling case: run only that pass (config 3's soft forward or backward, or the MINIROCKET "
-                         "transform with 9,996 features) on 12 examples, three times, and exit")
+    ap.add_argument("--profile-pass", choices=["soft", "backward", "minirocket", "f16"], default=None,
+                    help="profiling case: run only that pass (config 3's soft forward or backward, the MINIROCKET "
+                         "transform with 9,996 features, or the hard transform in half precision) on 12 examples, "
+                         "three times, and exit")
     ap.add_argument("--gemm-probe", action="store_true",
                     help="measure what a library GEMM makes of the zero-padded dense-channel formulation of the transform "
                          "(a reference measurement for the design notes: the transform itself never calls a GEMM) and exit")
@@ -326,6 +327,17 @@ def main():
             e1.record()
             torch.cuda.synchronize()
             print(json.dumps({"pass": "minirocket", "shape": "N=12 x C=%d x L=%d, %d features" % (w["C"], w["L"], MINI_FEATURES),
+                              "ms": e0.elapsed_time(e1) / 2}))
+            return
+        if args.profile_pass == "f16":
+            hfeat = rk.rocket_transform_f16(params, Xs)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(2):
+                rk.rocket_transform_f16(params, Xs, out=hfeat)
+            e1.record()
+            torch.cuda.synchronize()
+            print(json.dumps({"pass": "f16", "shape": "N=12 x C=%d x L=%d, K=%d" % (w["C"], w["L"], w["K"]),
                               "ms": e0.elapsed_time(e1) / 2}))
             return
         sfeat, arg = rk.rocket_transform_soft(params, Xs, LAMBDA, SHIFT)
